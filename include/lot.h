@@ -1,0 +1,152 @@
+/*
+ * lot.h -- C ABI of liblot: the forward hot path of LOTFormer attention
+ * (arXiv 2509.23436, Section "Method") as hand-written CUDA for sm_100a.
+ *
+ * For each (batch b, head h) slice, with queries/keys/values q,k,v [n,d], pivot
+ * locations z_h [r,d] and pivot masses beta_h [r] (> 0, summing to 1):
+ *
+ *   costs        C1[i,t] = <q_i, z_t>,  C2[j,t] = <k_j, z_t>            (display after
+ *                "Setting similarity to c(q,k) = q^T k"; no 1/sqrt(d) factor)
+ *   two solves   Gamma1 in U(beta, a), Gamma2 in U(beta, b), the entropic problems
+ *                Eq. (1)-(2), in the Sinkhorn scaling form Diag(u) exp(C/eps) Diag(v)
+ *   composition  Gamma = Gamma1^T Diag(beta)^-1 Gamma2 (Eq. (3)), never formed
+ *   output       out = A V = Gamma1^T (Diag(beta)^-1 (Gamma2 V)) with A = Gamma / a the
+ *                row-stochastic scaling (A = n Gamma for uniform marginals; Eq. (4) and
+ *                the paragraph "Rank and complexity")
+ *
+ * The Sinkhorn map that every entry point computes (T = iters), per side with token
+ * marginal m (a for queries, b for keys):
+ *       g <- 0;  repeat T times:
+ *           f_i = eps (log m_i - LSE_t((C_it + g_t)/eps))
+ *           g_t = eps (log beta_t - LSE_i((C_it + f_i)/eps))
+ *       one closing update of f;  P_it = exp((C_it + f_i + g_t)/eps).
+ * Marginals: a_i = 1/n.  b_j = 1/n, or with a key length L_b: b_j = 1/L_b for j < L_b
+ * and tokens j >= L_b carry no mass (they take no part in the key-side problem).
+ *
+ * General conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says
+ *     "host".  Tensors are dense row-major, last index fastest, 16-byte aligned.
+ *   - q,k,v,out: [B,H,n,d] in `dtype` (LOT_F32 or LOT_BF16).  z: [H,r,d] float32,
+ *     beta: [H,r] float32, per head and shared over the batch.  key_len: [B] int32.
+ *   - Supported: B,H >= 1, n >= 1 (n*r, n*d < 2^31), 1 <= r <= 256, 8 <= d <= 256 with
+ *     d % 8 == 0, eps > 0 finite, iters >= 0.  B == 0 or n == 0 is a no-op returning
+ *     LOT_OK.  Anything else returns LOT_ERR_INVALID_ARG / LOT_ERR_UNSUPPORTED_SHAPE
+ *     before any launch.
+ *   - Calls are asynchronous on `stream` (NULL = the default stream), never
+ *     synchronise the host, never abort.  The return value reports argument and launch
+ *     errors only.  Conditions found on the device (a non-finite potential, an empty
+ *     key set) are OR-ed into a status word at the start of the workspace; read it
+ *     with lot_device_status after the work has run.
+ *   - Scratch memory comes from the caller (`ws`, `ws_bytes`; size from the matching
+ *     *_workspace_bytes call, 256-byte aligned).  The library keeps no state between
+ *     calls except inside lot_attention_fwd (see there).  Two calls may run
+ *     concurrently only on different workspaces.
+ *   - Results are deterministic: reductions across thread blocks are summed in a
+ *     fixed order, no floating-point atomics.
+ */
+#ifndef LOT_H_
+#define LOT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *lot_stream_t; /* a cudaStream_t */
+
+#if defined(__GNUC__)
+#define LOT_API __attribute__((visibility("default")))
+#else
+#define LOT_API
+#endif
+
+enum lot_status {
+    LOT_OK = 0,
+    LOT_ERR_INVALID_ARG = 1,       /* null pointer, misaligned pointer, eps <= 0, iters < 0, bad dtype */
+    LOT_ERR_UNSUPPORTED_SHAPE = 2, /* a size outside the supported set above */
+    LOT_ERR_WORKSPACE = 3,         /* ws null/misaligned or ws_bytes too small */
+    LOT_ERR_CUDA = 4               /* a CUDA runtime call or launch failed (cudaGetLastError consumed) */
+};
+
+enum lot_dtype { LOT_F32 = 0, LOT_BF16 = 1 };
+
+/* bits of the device status word */
+enum lot_device_flag {
+    LOT_DEV_NONFINITE = 1, /* a pivot potential became inf/nan (e.g. beta_t <= 0) */
+    LOT_DEV_EMPTY = 2,     /* a key_len entry was <= 0: that slice has no key mass; its output is zeros */
+    LOT_DEV_TIMEOUT = 4    /* a bounded device-side wait gave up; results of the call are invalid */
+};
+
+/* Library version: major*10000 + minor*100 + patch. */
+LOT_API int lot_version(void);
+
+/* Static string for a lot_status value (never NULL). */
+LOT_API const char *lot_status_string(int status);
+
+/*
+ * lot_cost -- the similarity matrices of Section "Method": cost[b,h,i,t] = <x[b,h,i,:], z[h,t,:]>.
+ *   x     [B,H,n,d] in `dtype`;  z [H,r,d] float32;  cost [B,H,n,r] float32 (out).
+ * float32 accumulation; bf16 inputs are used exactly.  Needs no workspace.
+ */
+LOT_API int lot_cost(const void *x, const float *z, int dtype, int B, int H, int n, int d, int r,
+             float *cost, lot_stream_t stream);
+
+/* Scratch bytes lot_sinkhorn needs for these sizes. */
+LOT_API size_t lot_sinkhorn_workspace_bytes(int B, int H, int n, int r);
+
+/*
+ * lot_sinkhorn -- one entropic solve, Eq. (1) or (2), from a materialised similarity matrix.
+ *   cost [B,H,n,r] float32;  beta [H,r];  len [B] int32 or NULL (tokens i >= len[b] carry
+ *   no mass and m_i = 1/len[b]; NULL means m_i = 1/n).
+ * Outputs (each may be NULL except g):
+ *   g    [B,H,r]   pivot potentials after T pivot updates (natural-log units, as above)
+ *   f    [B,H,n]   token potentials after the closing update (-inf for massless tokens)
+ *   plan [B,H,n,r] P_it (zero rows for massless tokens)
+ */
+LOT_API int lot_sinkhorn(const float *cost, const float *beta, const int32_t *len,
+                 int B, int H, int n, int r, float eps, int iters,
+                 float *g, float *f, float *plan,
+                 void *ws, size_t ws_bytes, lot_stream_t stream);
+
+/* Scratch bytes lot_attention_fwd_ex needs for these sizes. */
+LOT_API size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype);
+
+/*
+ * lot_attention_fwd_ex -- the whole forward path, Eq. (1)-(4): costs, both solves, apply.
+ *   q,k,v,out [B,H,n,d] in `dtype`;  z [H,r,d];  beta [H,r];  key_len [B] or NULL.
+ *   g1_out, g2_out [B,H,r] float32 or NULL: the final pivot potentials of the query-side
+ *   and key-side solves (natural-log units).
+ * out[b,h,i,:] = sum_t softmax_t((C1_it + g1_t)/eps) * W'_t,  W' = Diag(beta)^-1 Gamma2 V.
+ * Padded query rows (there is no query mask) produce ordinary finite outputs.
+ */
+LOT_API int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
+                         const float *z, const float *beta, const int32_t *key_len,
+                         int dtype, int B, int H, int n, int d, int r, float eps, int iters,
+                         void *out, float *g1_out, float *g2_out,
+                         void *ws, size_t ws_bytes, lot_stream_t stream);
+
+/*
+ * lot_attention_fwd -- the same path for float32 tensors, uniform marginals, with scratch the
+ * library manages itself: one buffer per device, grown with cudaMalloc when a call needs
+ * more than any earlier one (that call synchronises the device once; later calls of the
+ * same or smaller size allocate nothing).  Calls on one device are serialised by the
+ * caller (they share that buffer).  Arguments as lot_attention_fwd_ex.
+ */
+LOT_API int lot_attention_fwd(const float *q, const float *k, const float *v,
+                      const float *z, const float *beta,
+                      int B, int H, int n, int d, int r, float eps, int iters,
+                      float *out, lot_stream_t stream);
+
+/*
+ * lot_device_status -- copy the device status word of workspace `ws` (as passed to
+ * lot_sinkhorn / lot_attention_fwd_ex; NULL = the library-managed buffer of the current
+ * device) to *status (host), after synchronising `stream`.  0 means nothing was flagged.
+ */
+LOT_API int lot_device_status(const void *ws, lot_stream_t stream, int *status /* host */);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOT_H_ */

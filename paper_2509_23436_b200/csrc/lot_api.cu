@@ -1,0 +1,289 @@
+// The C ABI of liblot (see include/lot.h): argument validation, workspace carving and the
+// launch sequence.  No arithmetic of the method lives here.
+#include "../../include/lot.h"
+#include "lot_internal.h"
+
+#include <math.h>
+#include <mutex>
+
+namespace {
+
+using namespace lot;
+
+constexpr int kMaxR = 256;
+constexpr int kMaxD = 256;
+constexpr int kMaxDevices = 64;
+
+inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_dims(int B, int H, int n, int r)
+{
+    if (B < 0 || H < 1 || n < 0 || r < 1) return LOT_ERR_INVALID_ARG;
+    if (r > kMaxR) return LOT_ERR_UNSUPPORTED_SHAPE;
+    if ((long long)B * H > 32767) return LOT_ERR_UNSUPPORTED_SHAPE;
+    if ((long long)n * r >= (1ll << 31)) return LOT_ERR_UNSUPPORTED_SHAPE;
+    return LOT_OK;
+}
+
+int check_d(int n, int d)
+{
+    if (d < 1) return LOT_ERR_INVALID_ARG;
+    if (d < 8 || d > kMaxD || (d % 8) != 0) return LOT_ERR_UNSUPPORTED_SHAPE;
+    if ((long long)n * d >= (1ll << 31)) return LOT_ERR_UNSUPPORTED_SHAPE;
+    return LOT_OK;
+}
+
+// Workspace of one Sinkhorn problem set.  The head (status word, potentials, tickets) is one
+// contiguous region cleared at the start of every call.
+struct SinkLayout {
+    size_t status, G, counter, head_end, gnat, part, M, total;
+    int chunks, rows_per_chunk;
+};
+
+// lt = bytes of the type potentials and row log-sum-exps are held in (4 or 8).
+SinkLayout sink_layout(int nprob, int n, int r, size_t base, size_t lt)
+{
+    SinkLayout L;
+    L.chunks = pass_chunks(nprob > 0 ? nprob : 1, n > 0 ? n : 1);
+    L.rows_per_chunk = (n + L.chunks - 1) / L.chunks;
+    size_t o = base;
+    L.status = o; o += 256;
+    L.G = o; o += up256((size_t)nprob * r * lt);
+    L.counter = o; o += up256((size_t)nprob * 4);
+    L.head_end = o;
+    L.gnat = o; o += up256((size_t)nprob * r * 4);
+    L.part = o; o += up256((size_t)nprob * L.chunks * r * 2 * 4);
+    L.M = o; o += up256((size_t)nprob * n * lt);
+    L.total = o;
+    return L;
+}
+
+struct AttnLayout {
+    SinkLayout s;
+    size_t counter2, cost, wpart, Wp, total;
+    int achunks, arows;
+};
+
+AttnLayout attn_layout(int B, int H, int n, int d, int r, int dtype)
+{
+    AttnLayout A;
+    const size_t lt = dtype == LOT_F32 ? 8 : 4;
+    const int BH = B * H;
+    // tickets of the apply stage sit right behind the status word so one memset clears all
+    size_t o = 0;
+    int tiles = ((r + 63) / 64) * ((d + 63) / 64) * BH;
+    A.counter2 = 256;
+    o = 256 + up256((size_t)tiles * 4);
+    A.s = sink_layout(2 * BH, n, r, o, lt);
+    A.s.status = 0; // shared status word at the very start
+    o = A.s.total;
+    A.cost = o; o += up256((size_t)2 * BH * n * r * lt);
+    A.achunks = apply_chunks(BH > 0 ? BH : 1, n > 0 ? n : 1, r, d);
+    A.arows = (n + A.achunks - 1) / A.achunks;
+    A.wpart = o; o += up256((size_t)BH * A.achunks * r * d * 4);
+    A.Wp = o; o += up256((size_t)BH * r * d * 4);
+    A.total = o;
+    return A;
+}
+
+template <typename T> inline T *at(void *ws, size_t off) { return reinterpret_cast<T *>(static_cast<char *>(ws) + off); }
+
+struct Managed {
+    void *ptr = nullptr;
+    size_t bytes = 0;
+};
+Managed g_managed[kMaxDevices];
+std::mutex g_managed_mu;
+
+} // namespace
+
+extern "C" {
+
+int lot_version(void) { return 100; }
+
+const char *lot_status_string(int status)
+{
+    switch (status) {
+    case LOT_OK: return "LOT_OK";
+    case LOT_ERR_INVALID_ARG: return "LOT_ERR_INVALID_ARG: null or misaligned pointer, eps <= 0, iters < 0 or unknown dtype";
+    case LOT_ERR_UNSUPPORTED_SHAPE: return "LOT_ERR_UNSUPPORTED_SHAPE: need 1 <= r <= 256, 8 <= d <= 256, d % 8 == 0, B*H <= 32767, n*r and n*d < 2^31";
+    case LOT_ERR_WORKSPACE: return "LOT_ERR_WORKSPACE: workspace null, not 256-byte aligned or too small";
+    case LOT_ERR_CUDA: return "LOT_ERR_CUDA: a CUDA runtime call or kernel launch failed";
+    default: return "unknown lot status";
+    }
+}
+
+int lot_cost(const void *x, const float *z, int dtype, int B, int H, int n, int d, int r,
+             float *cost, lot_stream_t stream)
+{
+    if (dtype != LOT_F32 && dtype != LOT_BF16) return LOT_ERR_INVALID_ARG;
+    int st = check_dims(B, H, n, r);
+    if (st != LOT_OK) return st;
+    st = check_d(n, d);
+    if (st != LOT_OK) return st;
+    if (B == 0 || n == 0) return LOT_OK;
+    if (!x || !z || !cost) return LOT_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(z) || !aligned16(cost)) return LOT_ERR_INVALID_ARG;
+    cudaError_t e = launch_cost(x, z, dtype, B * H, H, n, d, r, cost, false, (cudaStream_t)stream);
+    return e == cudaSuccess ? LOT_OK : LOT_ERR_CUDA;
+}
+
+size_t lot_sinkhorn_workspace_bytes(int B, int H, int n, int r)
+{
+    if (check_dims(B, H, n, r) != LOT_OK) return 0;
+    return sink_layout(B * H, n, r, 0, 8).total;
+}
+
+int lot_sinkhorn(const float *cost, const float *beta, const int32_t *len,
+                 int B, int H, int n, int r, float eps, int iters,
+                 float *g, float *f, float *plan,
+                 void *ws, size_t ws_bytes, lot_stream_t stream)
+{
+    int st = check_dims(B, H, n, r);
+    if (st != LOT_OK) return st;
+    if (!(eps > 0.f) || !isfinite(eps) || iters < 0) return LOT_ERR_INVALID_ARG;
+    if (B == 0 || n == 0) return LOT_OK;
+    if (!cost || !beta || !g) return LOT_ERR_INVALID_ARG;
+    if (!aligned16(cost) || !aligned16(beta) || !aligned16(g) || !aligned16(f) || !aligned16(plan) ||
+        (len && (reinterpret_cast<uintptr_t>(len) & 3u)))
+        return LOT_ERR_INVALID_ARG;
+    const int nprob = B * H;
+    SinkLayout L = sink_layout(nprob, n, r, 0, 8);
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < L.total) return LOT_ERR_WORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(ws, 0, L.head_end, s) != cudaSuccess) return LOT_ERR_CUDA;
+
+    PassArgs a{};
+    a.cost = cost; a.beta = beta; a.len = len; a.len_from = 0;
+    a.G = at<void>(ws, L.G); a.part = at<float>(ws, L.part); a.counter = at<unsigned>(ws, L.counter);
+    a.M = at<void>(ws, L.M); a.g_out = g; a.f_out = f; a.plan_out = plan;
+    a.status = at<int>(ws, L.status);
+    a.nprob = nprob; a.B = B; a.H = H; a.n = n; a.r = r;
+    a.chunks = L.chunks; a.rows_per_chunk = L.rows_per_chunk;
+    a.mode = kModeCostF32Wide;
+    a.scale_d = 1.4426950408889634 / (double)eps;
+    a.eps_ln2 = (float)((double)eps * 0.6931471805599453);
+    for (int it = 0; it < iters; ++it)
+        if (launch_sinkhorn_pass(a, false, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_sinkhorn_pass(a, true, s) != cudaSuccess) return LOT_ERR_CUDA;
+    return LOT_OK;
+}
+
+size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype)
+{
+    if (dtype != LOT_F32 && dtype != LOT_BF16) return 0;
+    if (check_dims(B, H, n, r) != LOT_OK || check_d(n, d) != LOT_OK) return 0;
+    return attn_layout(B, H, n, d, r, dtype).total;
+}
+
+int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
+                         const float *z, const float *beta, const int32_t *key_len,
+                         int dtype, int B, int H, int n, int d, int r, float eps, int iters,
+                         void *out, float *g1_out, float *g2_out,
+                         void *ws, size_t ws_bytes, lot_stream_t stream)
+{
+    if (dtype != LOT_F32 && dtype != LOT_BF16) return LOT_ERR_INVALID_ARG;
+    int st = check_dims(B, H, n, r);
+    if (st != LOT_OK) return st;
+    st = check_d(n, d);
+    if (st != LOT_OK) return st;
+    if (!(eps > 0.f) || !isfinite(eps) || iters < 0) return LOT_ERR_INVALID_ARG;
+    if (B == 0 || n == 0) return LOT_OK;
+    if (!q || !k || !v || !z || !beta || !out) return LOT_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(z) || !aligned16(beta) ||
+        !aligned16(out) || !aligned16(g1_out) || !aligned16(g2_out) ||
+        (key_len && (reinterpret_cast<uintptr_t>(key_len) & 3u)))
+        return LOT_ERR_INVALID_ARG;
+    AttnLayout A = attn_layout(B, H, n, d, r, dtype);
+    const bool wide = dtype == LOT_F32;
+    const size_t lt = wide ? 8 : 4;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < A.total) return LOT_ERR_WORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int BH = B * H;
+    if (cudaMemsetAsync(ws, 0, A.s.head_end, s) != cudaSuccess) return LOT_ERR_CUDA;
+
+    char *cost1 = at<char>(ws, A.cost);
+    char *cost2 = cost1 + (size_t)BH * n * r * lt;
+    if (launch_cost(q, z, dtype, BH, H, n, d, r, cost1, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_cost(k, z, dtype, BH, H, n, d, r, cost2, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+
+    PassArgs a{};
+    a.cost = cost1; a.beta = beta; a.len = key_len; a.len_from = BH;
+    a.G = at<void>(ws, A.s.G); a.part = at<float>(ws, A.s.part); a.counter = at<unsigned>(ws, A.s.counter);
+    a.M = at<void>(ws, A.s.M); a.g_out = at<float>(ws, A.s.gnat); a.f_out = nullptr; a.plan_out = nullptr;
+    a.status = at<int>(ws, 0);
+    a.nprob = 2 * BH; a.B = B; a.H = H; a.n = n; a.r = r;
+    a.chunks = A.s.chunks; a.rows_per_chunk = A.s.rows_per_chunk;
+    a.mode = wide ? kModeWide : kModeF32;
+    a.scale_d = 1.4426950408889634 / (double)eps;
+    a.eps_ln2 = (float)((double)eps * 0.6931471805599453);
+    for (int it = 0; it < iters; ++it)
+        if (launch_sinkhorn_pass(a, false, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_sinkhorn_pass(a, true, s) != cudaSuccess) return LOT_ERR_CUDA;
+
+    ApplyArgs ap{};
+    ap.cost1 = cost1; ap.cost2 = cost2;
+    ap.G1 = a.G; ap.G2 = static_cast<char *>(a.G) + (size_t)BH * r * lt;
+    ap.M1 = a.M; ap.M2 = static_cast<char *>(a.M) + (size_t)BH * n * lt;
+    ap.beta = beta; ap.key_len = key_len; ap.v = v; ap.out = out;
+    ap.wpart = at<float>(ws, A.wpart); ap.Wp = at<float>(ws, A.Wp); ap.counter = at<unsigned>(ws, A.counter2);
+    ap.B = B; ap.H = H; ap.n = n; ap.d = d; ap.r = r;
+    ap.chunks = A.achunks; ap.rows_per_chunk = A.arows; ap.scale_d = a.scale_d;
+    if (launch_apply_w(ap, dtype, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_apply_out(ap, dtype, s) != cudaSuccess) return LOT_ERR_CUDA;
+
+    const size_t gb = (size_t)BH * r * sizeof(float);
+    if (g1_out && cudaMemcpyAsync(g1_out, a.g_out, gb, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (g2_out && cudaMemcpyAsync(g2_out, a.g_out + (size_t)BH * r, gb, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return LOT_ERR_CUDA;
+    return LOT_OK;
+}
+
+int lot_attention_fwd(const float *q, const float *k, const float *v,
+                      const float *z, const float *beta,
+                      int B, int H, int n, int d, int r, float eps, int iters,
+                      float *out, lot_stream_t stream)
+{
+    int st = check_dims(B, H, n, r);
+    if (st != LOT_OK) return st;
+    st = check_d(n, d);
+    if (st != LOT_OK) return st;
+    if (B == 0 || n == 0) return LOT_OK;
+    const size_t need = attn_layout(B, H, n, d, r, LOT_F32).total;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LOT_ERR_CUDA;
+    void *ws = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_managed_mu);
+        Managed &m = g_managed[dev];
+        if (m.bytes < need) {
+            if (cudaDeviceSynchronize() != cudaSuccess) return LOT_ERR_CUDA;
+            if (m.ptr) cudaFree(m.ptr);
+            m.ptr = nullptr; m.bytes = 0;
+            if (cudaMalloc(&m.ptr, need) != cudaSuccess) { (void)cudaGetLastError(); m.ptr = nullptr; return LOT_ERR_CUDA; }
+            m.bytes = need;
+        }
+        ws = m.ptr;
+    }
+    return lot_attention_fwd_ex(q, k, v, z, beta, nullptr, LOT_F32, B, H, n, d, r, eps, iters,
+                                out, nullptr, nullptr, ws, need, stream);
+}
+
+int lot_device_status(const void *ws, lot_stream_t stream, int *status)
+{
+    if (!status) return LOT_ERR_INVALID_ARG;
+    if (!ws) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LOT_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(g_managed_mu);
+        ws = g_managed[dev].ptr;
+        if (!ws) { *status = 0; return LOT_OK; }
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(status, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return LOT_ERR_CUDA;
+    return LOT_OK;
+}
+
+} // extern "C"

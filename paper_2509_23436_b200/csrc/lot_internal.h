@@ -1,0 +1,65 @@
+// Internal launch interface between the C ABI (lot_api.cu) and the kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace lot {
+
+// One Sinkhorn pass over a set of independent problems.  Problem p covers the slice
+// s = p % (B*H) (batch s / H, head s % H); problems p >= len_from take their valid length
+// from len[batch], the others use n.
+// Arithmetic modes: which types the similarity matrix is stored in and the logits, pivot
+// potentials G and row log-sum-exps M are assembled in.
+enum { kModeF32 = 0,          // cost float, logits float            (bf16 tensors)
+       kModeCostF32Wide = 1,  // cost float, logits/G/M double       (lot_sinkhorn)
+       kModeWide = 2 };       // cost double, logits/G/M double      (float32 tensors)
+
+struct PassArgs {
+    const void *cost;    // [nprob][n][r] similarity matrices (float or double, see mode)
+    const float *beta;   // [H][r]
+    const int32_t *len;  // [B] or nullptr
+    int len_from;
+    void *G;             // [nprob][r] pivot potentials, base-2 log units (in/out; float or double)
+    float *part;         // [nprob][chunks][r][2] per-block column pairs (kappa, S)
+    unsigned *counter;   // [nprob] arrival tickets, zero on entry and on exit
+    void *M;             // final pass: [nprob][n] row log-sum-exp (base 2), +inf for massless rows
+    float *g_out;        // final pass, optional: [nprob][r] potentials in natural-log units
+    float *f_out;        // final pass, optional: [nprob][n]
+    float *plan_out;     // final pass, optional: [nprob][n][r]
+    int *status;
+    int nprob, B, H, n, r;
+    int chunks, rows_per_chunk;
+    int mode;
+    double scale_d;      // log2(e)/eps
+    float eps_ln2;       // eps*ln(2)
+};
+
+struct ApplyArgs {
+    const void *cost1;   // [BH][n][r] query-side similarities (float: bf16 tensors, double: float32)
+    const void *cost2;   // [BH][n][r] key-side similarities
+    const void *G1, *G2;   // [BH][r]   same type as the similarities
+    const void *M1, *M2;   // [BH][n]
+    const float *beta;     // [H][r]
+    const int32_t *key_len;
+    const void *v;         // [BH][n][d]
+    void *out;             // [BH][n][d]
+    float *wpart;          // [BH][chunks][r][d]
+    float *Wp;             // [BH][r][d]  W' = Diag(beta)^-1 Gamma2 V
+    unsigned *counter;     // [BH * tblks * cblks]
+    int B, H, n, d, r;
+    int chunks, rows_per_chunk;
+    double scale_d;
+};
+
+int pass_chunks(int nprob, int n);
+int apply_chunks(int BH, int n, int r, int d);
+
+cudaError_t launch_cost(const void *x, const float *z, int dtype, int BH, int H, int n, int d, int r,
+                        void *cost, bool wide, cudaStream_t st);
+cudaError_t launch_sinkhorn_pass(const PassArgs &a, bool final_pass, cudaStream_t st);
+cudaError_t launch_apply_w(const ApplyArgs &a, int dtype, cudaStream_t st);
+cudaError_t launch_apply_out(const ApplyArgs &a, int dtype, cudaStream_t st);
+
+} // namespace lot

@@ -1,0 +1,477 @@
+// General (any supported shape, float32 or bf16 tensors) kernels of the LOT attention
+// forward path: similarity matrices, Sinkhorn passes over a materialised similarity
+// matrix, and the two apply stages of Eq. (4).  All arithmetic is float32 on the CUDA
+// cores; cross-block reductions are per-block partials summed in a fixed order by the
+// last block to arrive (no spinning, no floating-point atomics).
+#include "lot_common.cuh"
+#include "lot_internal.h"
+
+namespace lot {
+
+// ------------------------------------------------------------------------------------
+// Similarity matrix C[i,t] = <x_i, z_t>  (Section "Method", dot-product similarity).
+// Block = 64 tokens x 64 pivots, 256 threads, 4x4 outputs per thread, K chunks of 32.
+// ------------------------------------------------------------------------------------
+constexpr int kTile = 64;
+constexpr int kTileK = 32;
+constexpr int kPadT = kTile + 4;
+
+template <typename T, typename AccT, typename OutT>
+__global__ void __launch_bounds__(256)
+cost_kernel(const T *__restrict__ x, const float *__restrict__ z, OutT *__restrict__ cost,
+            int H, int n, int d, int r)
+{
+    __shared__ __align__(16) AccT Xs[kTileK][kPadT];
+    __shared__ __align__(16) AccT Zs[kTileK][kPadT];
+    const int bh = blockIdx.z, h = bh % H;
+    const int i0 = blockIdx.x * kTile, t0 = blockIdx.y * kTile;
+    const T *xb = x + (size_t)bh * n * d;
+    const float *zb = z + (size_t)h * r * d;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    AccT acc[4][4] = {};
+    for (int k0 = 0; k0 < d; k0 += kTileK) {
+#pragma unroll
+        for (int rep = 0; rep < 2; ++rep) {
+            int idx = threadIdx.x + rep * 256;
+            int row = idx / 8, k4 = (idx % 8) * 4;
+            float xv[4] = {0.f, 0.f, 0.f, 0.f}, zv[4] = {0.f, 0.f, 0.f, 0.f};
+            if (i0 + row < n && k0 + k4 < d) load4(xb + (size_t)(i0 + row) * d + k0 + k4, xv);
+            if (t0 + row < r && k0 + k4 < d) load4(zb + (size_t)(t0 + row) * d + k0 + k4, zv);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                Xs[k4 + j][row] = (AccT)xv[j];
+                Zs[k4 + j][row] = (AccT)zv[j];
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < kTileK; ++kk) {
+            AccT xr[4], zr[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) { xr[a] = Xs[kk][ty * 4 + a]; zr[a] = Zs[kk][tx * 4 + a]; }
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] = fma(xr[a], zr[b], acc[a][b]);
+        }
+        __syncthreads();
+    }
+    OutT *cb = cost + (size_t)bh * n * r;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        int i = i0 + ty * 4 + a;
+        if (i >= n) continue;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            int t = t0 + tx * 4 + b;
+            if (t < r) cb[(size_t)i * r + t] = (OutT)acc[a][b];
+        }
+    }
+}
+
+// float32 tensors: exact products accumulated in float64 (the logits C/eps amplify the
+// similarity error by 1/eps); bf16 tensors: float32 accumulation.  `wide` selects a float64
+// result (the attention path's internal similarity matrix for float32 tensors).
+cudaError_t launch_cost(const void *x, const float *z, int dtype, int BH, int H, int n, int d, int r,
+                        void *cost, bool wide, cudaStream_t st)
+{
+    dim3 grid((n + kTile - 1) / kTile, (r + kTile - 1) / kTile, BH);
+    if (dtype == 0) {
+        const float *xf = static_cast<const float *>(x);
+        if (wide) cost_kernel<float, double, double><<<grid, 256, 0, st>>>(xf, z, static_cast<double *>(cost), H, n, d, r);
+        else cost_kernel<float, double, float><<<grid, 256, 0, st>>>(xf, z, static_cast<float *>(cost), H, n, d, r);
+    } else {
+        cost_kernel<__nv_bfloat16, float, float><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(x), z,
+                                                                        static_cast<float *>(cost), H, n, d, r);
+    }
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------
+// One Sinkhorn pass (Eq. (1)-(2), scaling form).  With the token potential eliminated,
+//   token update : M_i = log2 sum_t 2^(L_it + G_t)                       (row log-sum-exp)
+//   pivot update : G_t += log2(beta_t / m) - log2 sum_i 2^(L_it + G_t - M_i)
+// where m = 1/n_valid is the token mass.  Rows are spread over GS lanes (GS = 8, 16 or
+// 32), each lane holding CPL columns t = lane + k*GS; row reductions are shuffles, column
+// sums are carried per lane as (kappa, S) pairs and merged lane -> warp -> block -> grid.
+// FINAL = closing token update: writes M (and optionally g, f, plan), no pivot update.
+// ------------------------------------------------------------------------------------
+constexpr int kPassWarps = 8;
+
+// CostT = stored similarity type, LT = type the logits, potentials and row LSE are assembled
+// in (float for bf16 tensors; double when the caller's tensors are float32, so that logits of
+// magnitude ~1e3 at small eps keep an absolute accuracy well below the 1e-4 output tolerance).
+template <int GS, int CPL, bool FINAL, typename CostT, typename LT>
+__global__ void __launch_bounds__(kPassWarps * 32)
+sinkhorn_pass_kernel(PassArgs a)
+{
+    __shared__ float sm_k[kPassWarps][256];
+    __shared__ float sm_s[kPassWarps][256];
+    __shared__ int sm_last;
+    const int p = blockIdx.x / a.chunks, chunk = blockIdx.x % a.chunks;
+    const int slice = p % (a.B * a.H), b = slice / a.H, h = slice % a.H;
+    int nvalid = a.n;
+    if (a.len != nullptr && p >= a.len_from) nvalid = min(max(a.len[b], 0), a.n);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int RPW = 32 / GS;
+    const int sub = lane / GS, cl = lane % GS;
+    const int r = a.r;
+    const CostT *C = static_cast<const CostT *>(a.cost) + (size_t)p * a.n * r;
+    LT *Gp = static_cast<LT *>(a.G) + (size_t)p * r;
+    LT *Mp = static_cast<LT *>(a.M) + (size_t)p * a.n;
+    const LT scale = (LT)a.scale_d;
+
+    LT Gk[CPL];
+    float kap[CPL], S[CPL];
+    bool cv[CPL];
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) {
+        int t = cl + k * GS;
+        cv[k] = t < r;
+        Gk[k] = cv[k] ? Gp[t] : (LT)0;
+        kap[k] = neg_inf();
+        S[k] = 0.f;
+    }
+    const int row0 = chunk * a.rows_per_chunk;
+    const int row_end = min(row0 + a.rows_per_chunk, a.n);       // rows this block owns
+    const int row1 = min(row_end, nvalid);                        // ... that carry mass
+    const int loop_end = FINAL ? row_end : row1;
+    const float log2m = -lg2((float)max(nvalid, 1));
+    const float mass = 1.f / (float)max(nvalid, 1);
+
+    for (int base = row0 + warp * RPW; base < loop_end; base += kPassWarps * RPW) {
+        const int i = base + sub;
+        const bool rv = i < row1;
+        LT l[CPL];
+        LT m = (LT)neg_inf();
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) {
+            LT c = (rv && cv[k]) ? (LT)__ldg(C + (size_t)i * r + cl + k * GS) : (LT)0;
+            l[k] = cv[k] ? fma(c, scale, Gk[k]) : (LT)neg_inf();
+            m = fmax(m, l[k]);
+        }
+#pragma unroll
+        for (int off = GS / 2; off > 0; off >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, off));
+        float e[CPL];
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) {
+            e[k] = (float)(l[k] - m);          // <= 0, exact difference of nearby logits
+            s += ex2(e[k]);
+        }
+#pragma unroll
+        for (int off = GS / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        const float lgs = lg2(s);
+        if (!FINAL) {
+            if (rv) {
+#pragma unroll
+                for (int k = 0; k < CPL; ++k)
+                    if (cv[k]) pair_add(kap[k], S[k], e[k] - lgs);
+            }
+        } else if (i < row_end) {
+            if (cl == 0) {
+                const LT Mi = m + (LT)lgs;
+                Mp[i] = rv ? Mi : (LT)__int_as_float(0x7f800000);
+                if (a.f_out) a.f_out[(size_t)p * a.n + i] = rv ? (float)((LT)a.eps_ln2 * ((LT)log2m - Mi)) : neg_inf();
+            }
+            if (a.plan_out) {
+#pragma unroll
+                for (int k = 0; k < CPL; ++k)
+                    if (cv[k])
+                        a.plan_out[((size_t)p * a.n + i) * r + cl + k * GS] = rv ? mass * ex2(e[k] - lgs) : 0.f;
+            }
+        }
+    }
+    if (FINAL) {
+        if (chunk == 0 && a.g_out != nullptr && threadIdx.x < r)
+            a.g_out[(size_t)p * r + threadIdx.x] = (float)(Gp[threadIdx.x] * (LT)a.eps_ln2);
+        return;
+    }
+
+    // lanes of different row groups hold the same columns: merge them, then the warps
+#pragma unroll
+    for (int off = GS; off < 32; off <<= 1) {
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) {
+            float k2 = __shfl_xor_sync(0xffffffffu, kap[k], off);
+            float s2 = __shfl_xor_sync(0xffffffffu, S[k], off);
+            pair_merge(kap[k], S[k], k2, s2);
+        }
+    }
+    if (sub == 0) {
+#pragma unroll
+        for (int k = 0; k < CPL; ++k)
+            if (cv[k]) {
+                sm_k[warp][cl + k * GS] = kap[k];
+                sm_s[warp][cl + k * GS] = S[k];
+            }
+    }
+    __syncthreads();
+    const int t = threadIdx.x;
+    if (t < r) {
+        float kk = sm_k[0][t], ss = sm_s[0][t];
+#pragma unroll
+        for (int w = 1; w < kPassWarps; ++w) pair_merge(kk, ss, sm_k[w][t], sm_s[w][t]);
+        float *dst = a.part + (((size_t)p * a.chunks + chunk) * r + t) * 2;
+        __stcg(dst, kk);
+        __stcg(dst + 1, ss);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned ticket = atomicAdd(a.counter + p, 1u);
+        sm_last = (ticket == (unsigned)a.chunks - 1u);
+    }
+    __syncthreads();
+    if (!sm_last) return;
+    __threadfence();
+    if (t < r) {
+        float kk = neg_inf(), ss = 0.f;
+        for (int c = 0; c < a.chunks; ++c) {
+            const float *src = a.part + (((size_t)p * a.chunks + c) * r + t) * 2;
+            pair_merge(kk, ss, __ldcg(src), __ldcg(src + 1));
+        }
+        if (nvalid <= 0) {
+            atomicOr(a.status, 2 /* LOT_DEV_EMPTY */);
+        } else {
+            LT lam = (LT)kk + (LT)lg2(ss);
+            LT gn = Gp[t] + (LT)lg2(a.beta[h * r + t] * (float)nvalid) - lam;
+            if (!isfinite((float)gn)) atomicOr(a.status, 1 /* LOT_DEV_NONFINITE */);
+            Gp[t] = gn;
+        }
+    }
+    if (threadIdx.x == 0) a.counter[p] = 0u;
+}
+
+int pass_chunks(int nprob, int n)
+{
+    // enough blocks for ~4 per SM over 148 SMs, at least 64 rows each
+    int want = (592 + nprob - 1) / nprob;
+    int most = (n + 63) / 64;
+    int c = want < most ? want : most;
+    return c < 1 ? 1 : c;
+}
+
+template <int GS, int CPL, typename CostT, typename LT>
+static cudaError_t launch_pass_t(const PassArgs &a, bool final_pass, cudaStream_t st)
+{
+    dim3 grid((unsigned)(a.nprob * a.chunks));
+    if (final_pass)
+        sinkhorn_pass_kernel<GS, CPL, true, CostT, LT><<<grid, kPassWarps * 32, 0, st>>>(a);
+    else
+        sinkhorn_pass_kernel<GS, CPL, false, CostT, LT><<<grid, kPassWarps * 32, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+template <typename CostT, typename LT>
+static cudaError_t launch_pass_r(const PassArgs &a, bool final_pass, cudaStream_t st)
+{
+    const int r = a.r;
+    if (r <= 8) return launch_pass_t<8, 1, CostT, LT>(a, final_pass, st);
+    if (r <= 16) return launch_pass_t<16, 1, CostT, LT>(a, final_pass, st);
+    if (r <= 32) return launch_pass_t<32, 1, CostT, LT>(a, final_pass, st);
+    if (r <= 64) return launch_pass_t<32, 2, CostT, LT>(a, final_pass, st);
+    if (r <= 128) return launch_pass_t<32, 4, CostT, LT>(a, final_pass, st);
+    return launch_pass_t<32, 8, CostT, LT>(a, final_pass, st);
+}
+
+cudaError_t launch_sinkhorn_pass(const PassArgs &a, bool final_pass, cudaStream_t st)
+{
+    switch (a.mode) {
+    case kModeF32: return launch_pass_r<float, float>(a, final_pass, st);
+    case kModeCostF32Wide: return launch_pass_r<float, double>(a, final_pass, st);
+    default: return launch_pass_r<double, double>(a, final_pass, st);
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Apply, key side (Eq. (4): Y = Gamma2 V, Z' = Diag(beta)^-1 Y).
+//   W'[t,c] = (1/beta_t) sum_j m 2^(L2_jt + G2_t - M2_j) v[j,c]
+// Block = 64 pivots x 64 channels over one chunk of keys; the last block of a tile sums
+// the chunk partials in order and scales.
+// ------------------------------------------------------------------------------------
+constexpr int kRowStep = 32;
+
+int apply_chunks(int BH, int n, int r, int d)
+{
+    int tiles = ((r + kTile - 1) / kTile) * ((d + kTile - 1) / kTile) * BH;
+    int want = (592 + tiles - 1) / tiles;
+    int most = (n + 255) / 256;
+    int c = want < most ? want : most;
+    return c < 1 ? 1 : c;
+}
+
+template <typename T, typename LT>
+__global__ void __launch_bounds__(256)
+apply_w_kernel(ApplyArgs a)
+{
+    __shared__ __align__(16) float Ps[kRowStep][kPadT];
+    __shared__ __align__(16) float Vs[kRowStep][kPadT];
+    __shared__ int sm_last;
+    const int bh = blockIdx.z, b = bh / a.H, h = bh % a.H;
+    const int cblks = (a.d + kTile - 1) / kTile;
+    const int tblk = blockIdx.y / cblks, cblk = blockIdx.y % cblks;
+    const int t0 = tblk * kTile, c0 = cblk * kTile;
+    const int chunk = blockIdx.x;
+    const int n = a.n, r = a.r, d = a.d;
+    int nvalid = n;
+    if (a.key_len != nullptr) nvalid = min(max(a.key_len[b], 0), n);
+    const int row0 = chunk * a.rows_per_chunk;
+    const int row1 = min(min(row0 + a.rows_per_chunk, n), nvalid);
+    const LT *C = static_cast<const LT *>(a.cost2) + (size_t)bh * n * r;
+    const LT *G = static_cast<const LT *>(a.G2) + (size_t)bh * r;
+    const LT *M = static_cast<const LT *>(a.M2) + (size_t)bh * n;
+    const LT scale = (LT)a.scale_d;
+    const T *V = static_cast<const T *>(a.v) + (size_t)bh * n * d;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    float acc[4][4] = {};
+
+    for (int j0 = row0; j0 < row1; j0 += kRowStep) {
+#pragma unroll
+        for (int rep = 0; rep < 8; ++rep) {
+            int idx = threadIdx.x + rep * 256;
+            int jj = idx / kTile, tt = idx % kTile;
+            int j = j0 + jj, t = t0 + tt;
+            float val = 0.f;
+            if (j < row1 && t < r) val = ex2((float)(fma(__ldg(C + (size_t)j * r + t), scale, __ldg(G + t)) - __ldg(M + j)));
+            Ps[jj][tt] = val;
+        }
+#pragma unroll
+        for (int rep = 0; rep < 2; ++rep) {
+            int idx = threadIdx.x + rep * 256;
+            int jj = idx / 16, c4 = (idx % 16) * 4;
+            int j = j0 + jj, c = c0 + c4;
+            float vv[4] = {0.f, 0.f, 0.f, 0.f};
+            if (j < row1 && c < d) load4(V + (size_t)j * d + c, vv);
+            *reinterpret_cast<float4 *>(&Vs[jj][c4]) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int jj = 0; jj < kRowStep; ++jj) {
+            float4 pa = *reinterpret_cast<const float4 *>(&Ps[jj][ty * 4]);
+            float4 vb = *reinterpret_cast<const float4 *>(&Vs[jj][tx * 4]);
+            float pr[4] = {pa.x, pa.y, pa.z, pa.w}, vr[4] = {vb.x, vb.y, vb.z, vb.w};
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y) acc[x][y] = fmaf(pr[x], vr[y], acc[x][y]);
+        }
+        __syncthreads();
+    }
+    float *wp = a.wpart + ((size_t)bh * a.chunks + chunk) * r * d;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        int t = t0 + ty * 4 + x;
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+            int c = c0 + tx * 4 + y;
+            if (t < r && c < d) __stcg(wp + (size_t)t * d + c, acc[x][y]);
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned ticket = atomicAdd(a.counter + (size_t)bh * gridDim.y + blockIdx.y, 1u);
+        sm_last = (ticket == (unsigned)a.chunks - 1u);
+    }
+    __syncthreads();
+    if (!sm_last) return;
+    __threadfence();
+    const float mass = nvalid > 0 ? 1.f / (float)nvalid : 0.f;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        int t = t0 + ty * 4 + x;
+        if (t >= r) continue;
+        const float sc = mass / a.beta[h * r + t];
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+            int c = c0 + tx * 4 + y;
+            if (c >= d) continue;
+            float sum = 0.f;
+            for (int ch = 0; ch < a.chunks; ++ch)
+                sum += __ldcg(a.wpart + (((size_t)bh * a.chunks + ch) * r + t) * d + c);
+            a.Wp[((size_t)bh * r + t) * d + c] = sum * sc;
+        }
+    }
+    if (threadIdx.x == 0) a.counter[(size_t)bh * gridDim.y + blockIdx.y] = 0u;
+}
+
+cudaError_t launch_apply_w(const ApplyArgs &a, int dtype, cudaStream_t st)
+{
+    int tblks = (a.r + kTile - 1) / kTile, cblks = (a.d + kTile - 1) / kTile;
+    dim3 grid(a.chunks, tblks * cblks, a.B * a.H);
+    if (dtype == 0) apply_w_kernel<float, double><<<grid, 256, 0, st>>>(a);
+    else apply_w_kernel<__nv_bfloat16, float><<<grid, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------
+// Apply, query side (Eq. (4): O = Gamma1^T Z', row-stochastic scaling):
+//   out[i,c] = sum_t 2^(L1_it + G1_t - M1_i) W'[t,c]
+// Block = 64 queries x 64 channels, pivots in steps of 32.
+// ------------------------------------------------------------------------------------
+template <typename T, typename LT>
+__global__ void __launch_bounds__(256)
+apply_out_kernel(ApplyArgs a)
+{
+    __shared__ __align__(16) float Ps[kTileK][kPadT];
+    __shared__ __align__(16) float Ws[kTileK][kPadT];
+    const int bh = blockIdx.z;
+    const int i0 = blockIdx.x * kTile, c0 = blockIdx.y * kTile;
+    const int n = a.n, r = a.r, d = a.d;
+    const LT *C = static_cast<const LT *>(a.cost1) + (size_t)bh * n * r;
+    const LT *G = static_cast<const LT *>(a.G1) + (size_t)bh * r;
+    const LT *M = static_cast<const LT *>(a.M1) + (size_t)bh * n;
+    const LT scale = (LT)a.scale_d;
+    const float *W = a.Wp + (size_t)bh * r * d;
+    T *O = static_cast<T *>(a.out) + (size_t)bh * n * d;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    float acc[4][4] = {};
+    for (int tb = 0; tb < r; tb += kTileK) {
+#pragma unroll
+        for (int rep = 0; rep < 8; ++rep) {
+            int idx = threadIdx.x + rep * 256;
+            int tt = idx % kTileK, ii = idx / kTileK;
+            int i = i0 + ii, t = tb + tt;
+            float val = 0.f;
+            if (i < n && t < r) val = ex2((float)(fma(__ldg(C + (size_t)i * r + t), scale, __ldg(G + t)) - __ldg(M + i)));
+            Ps[tt][ii] = val;
+        }
+#pragma unroll
+        for (int rep = 0; rep < 2; ++rep) {
+            int idx = threadIdx.x + rep * 256;
+            int tt = idx / 16, c4 = (idx % 16) * 4;
+            int t = tb + tt, c = c0 + c4;
+            float4 w = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (t < r && c < d) w = *reinterpret_cast<const float4 *>(W + (size_t)t * d + c);
+            *reinterpret_cast<float4 *>(&Ws[tt][c4]) = w;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int tt = 0; tt < kTileK; ++tt) {
+            float4 pa = *reinterpret_cast<const float4 *>(&Ps[tt][ty * 4]);
+            float4 wb = *reinterpret_cast<const float4 *>(&Ws[tt][tx * 4]);
+            float pr[4] = {pa.x, pa.y, pa.z, pa.w}, wr[4] = {wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y) acc[x][y] = fmaf(pr[x], wr[y], acc[x][y]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        int i = i0 + ty * 4 + x, c = c0 + tx * 4;
+        if (i < n && c < d) store4(O + (size_t)i * d + c, acc[x]);
+    }
+}
+
+cudaError_t launch_apply_out(const ApplyArgs &a, int dtype, cudaStream_t st)
+{
+    dim3 grid((a.n + kTile - 1) / kTile, (a.d + kTile - 1) / kTile, a.B * a.H);
+    if (dtype == 0) apply_out_kernel<float, double><<<grid, 256, 0, st>>>(a);
+    else apply_out_kernel<__nv_bfloat16, float><<<grid, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+} // namespace lot

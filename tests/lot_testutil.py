@@ -1,0 +1,65 @@
+"""Shared helpers of the parity tests: run the CUDA path through the C ABI, run the CPU oracle on
+chosen (batch, head) slices, and the error measure the tolerances are stated in."""
+import numpy as np
+import torch
+
+from oracle import lot_oracle as O
+from paper_2509_23436_b200 import binding as lot
+
+TOL = {torch.float32: 1e-4, torch.bfloat16: 2e-2}
+
+
+def to_dev(x):
+    dev = torch.device("cuda:0")
+    kl = None if x.key_len is None else x.key_len.to(dev)
+    return dict(q=x.q.to(dev), k=x.k.to(dev), v=x.v.to(dev), z=x.z.to(dev), beta=x.beta.to(dev), key_len=kl)
+
+
+def gpu_forward(x, want_g=False):
+    t = to_dev(x)
+    B, H, n, d, r = x.shape
+    g1 = torch.empty(B, H, r, device="cuda:0") if want_g else None
+    g2 = torch.empty(B, H, r, device="cuda:0") if want_g else None
+    out, ws = lot.lot_attention_fwd_ex(t["q"], t["k"], t["v"], t["z"], t["beta"], t["key_len"], x.eps, x.iters,
+                                       g1_out=g1, g2_out=g2)
+    torch.cuda.synchronize()
+    status = lot.lot_device_status(ws)
+    res = dict(out=out.float().cpu().double().numpy(), status=status)
+    if want_g:
+        res["g1"] = g1.cpu().double().numpy()
+        res["g2"] = g2.cpu().double().numpy()
+    return res
+
+
+def oracle_slice(x, b, h, return_potentials=False):
+    """Oracle output of one (batch, head) slice, from the rounded inputs."""
+    d = x.f64()
+    kl = None if d["key_len"] is None else d["key_len"][b:b + 1]
+    res = O.attention_fwd(d["q"][b:b + 1, h:h + 1], d["k"][b:b + 1, h:h + 1], d["v"][b:b + 1, h:h + 1],
+                          d["z"][h:h + 1], d["beta"][h:h + 1], x.eps, x.iters, key_len=kl,
+                          return_potentials=return_potentials)
+    if return_potentials:
+        return res[0][0, 0], res[1][0, 0], res[2][0, 0]
+    return res[0, 0]
+
+
+def oracle_all(x):
+    d = x.f64()
+    return O.attention_fwd(d["q"], d["k"], d["v"], d["z"], d["beta"], x.eps, x.iters, key_len=d["key_len"])
+
+
+def head_err(got, ref):
+    """max |got - ref| / max |ref| over one (batch, head) slice: the measure the tolerances
+    (1e-4 for float32 tensors, 2e-2 for bf16 tensors) are gated on."""
+    return float(np.abs(got - ref).max() / np.abs(ref).max())
+
+
+def worst_head_err(got, ref):
+    B, H = ref.shape[:2]
+    return max(head_err(got[b, h], ref[b, h]) for b in range(B) for h in range(H))
+
+
+def elem_err(got, ref, tol):
+    """Elementwise relative error with the absolute floor tol * rms(ref) (reported, not gated)."""
+    floor = tol * float(np.sqrt((ref ** 2).mean()))
+    return float((np.abs(got - ref) / np.maximum(np.abs(ref), floor / tol)).max())
