@@ -114,6 +114,14 @@ LOT_API int lot_sinkhorn(const float *cost, const float *beta, const int32_t *le
 LOT_API size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype);
 
 /*
+ * lot_launch_count -- how many kernels of this library one lot_attention_fwd_ex call with these
+ * parameters launches (host arithmetic only; 0 for iters < 0).  bf16 tensors with d = 64 and
+ * r <= 64 take the fused tensor-core path (similarities recomputed per pass from the tokens,
+ * never stored); every other supported shape takes the general path.
+ */
+LOT_API int lot_launch_count(int dtype, int d, int r, int iters);
+
+/*
  * lot_attention_fwd_ex -- the whole forward path, Eq. (1)-(4): costs, both solves, apply.
  *   q,k,v,out [B,H,n,d] in `dtype`;  z [H,r,d];  beta [H,r];  key_len [B] or NULL.
  *   g1_out, g2_out [B,H,r] float32 or NULL: the final pivot potentials of the query-side

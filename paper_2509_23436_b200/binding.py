@@ -30,6 +30,7 @@ SIGNATURES = {
     "lot_sinkhorn_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "lot_sinkhorn": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lot_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
+    "lot_launch_count": (_i, [_i, _i, _i, _i]),
     "lot_attention_fwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
                                   _vp, _vp, _vp, _vp, _sz, _vp]),
     "lot_attention_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp]),
@@ -127,6 +128,10 @@ def lot_sinkhorn(cost, beta, length, eps, iters, *, want_f=False, want_plan=Fals
 
 def lot_workspace_bytes(B, H, n, d, r, dtype_code) -> int:
     return lib().lot_workspace_bytes(B, H, n, d, r, dtype_code)
+
+
+def lot_launch_count(dtype_code: int, d: int, r: int, iters: int) -> int:
+    return lib().lot_launch_count(dtype_code, d, r, iters)
 
 
 def lot_attention_fwd_ex(q, k, v, z, beta, key_len, eps, iters, *, out=None, g1_out=None, g2_out=None,

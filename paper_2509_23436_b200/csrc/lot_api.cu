@@ -174,7 +174,15 @@ size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype)
 {
     if (dtype != LOT_F32 && dtype != LOT_BF16) return 0;
     if (check_dims(B, H, n, r) != LOT_OK || check_d(n, d) != LOT_OK) return 0;
+    if (fused_supported(dtype, d, r)) return fused_layout(B, H, n, d, r).total;
     return attn_layout(B, H, n, d, r, dtype).total;
+}
+
+int lot_launch_count(int dtype, int d, int r, int iters)
+{
+    if (iters < 0) return 0;
+    if (fused_supported(dtype, d, r)) return fused_launches(iters);
+    return 2 + iters + 1 + 2;
 }
 
 int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
@@ -195,6 +203,13 @@ int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
         !aligned16(out) || !aligned16(g1_out) || !aligned16(g2_out) ||
         (key_len && (reinterpret_cast<uintptr_t>(key_len) & 3u)))
         return LOT_ERR_INVALID_ARG;
+    if (fused_supported(dtype, d, r)) {
+        const size_t need = fused_layout(B, H, n, d, r).total;
+        if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < need) return LOT_ERR_WORKSPACE;
+        cudaError_t e = fused_attention(q, k, v, z, beta, key_len, B, H, n, d, r, eps, iters, out, g1_out, g2_out,
+                                        ws, (cudaStream_t)stream);
+        return e == cudaSuccess ? LOT_OK : LOT_ERR_CUDA;
+    }
     AttnLayout A = attn_layout(B, H, n, d, r, dtype);
     const bool wide = dtype == LOT_F32;
     const size_t lt = wide ? 8 : 4;

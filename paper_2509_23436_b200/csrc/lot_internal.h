@@ -62,4 +62,16 @@ cudaError_t launch_sinkhorn_pass(const PassArgs &a, bool final_pass, cudaStream_
 cudaError_t launch_apply_w(const ApplyArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_apply_out(const ApplyArgs &a, int dtype, cudaStream_t st);
 
+// ---- fused tensor-core path (lot_fused.cu): bf16 tensors, d = 64, r <= 64 ----
+struct FusedLayout {
+    size_t status, G, ticket, iter, robust, wticket, gnat, Wb, head_end, zprep, part, wpart, total;
+};
+bool fused_supported(int dtype, int d, int r);
+void fused_geometry(int B, int H, int n, int *q, int *ctas, int *maxslots);
+FusedLayout fused_layout(int B, int H, int n, int d, int r);
+cudaError_t fused_attention(const void *q, const void *k, const void *v, const float *z, const float *beta,
+                            const int32_t *key_len, int B, int H, int n, int d, int r, float eps, int iters,
+                            void *out, float *g1_out, float *g2_out, void *ws, cudaStream_t st);
+int fused_launches(int iters);
+
 } // namespace lot

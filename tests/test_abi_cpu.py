@@ -30,10 +30,13 @@ def test_exports_every_declared_symbol(L):
 
 
 def test_workspace_queries_are_host_only(L):
-    a = L.lot_workspace_bytes(1, 16, 16384, 64, 64, lot.LOT_BF16)
-    b = L.lot_workspace_bytes(1, 16, 65536, 64, 64, lot.LOT_BF16)
+    a = L.lot_workspace_bytes(1, 16, 16384, 64, 64, lot.LOT_F32)
+    b = L.lot_workspace_bytes(1, 16, 65536, 64, 64, lot.LOT_F32)
     assert 0 < a < b
     assert a % 256 == 0
+    # the fused bf16 path stores no similarity matrix: its scratch is far smaller
+    assert 0 < L.lot_workspace_bytes(1, 16, 16384, 64, 64, lot.LOT_BF16) < a // 8
+    assert L.lot_launch_count(lot.LOT_BF16, 64, 64, 10) > 0 and L.lot_launch_count(lot.LOT_F32, 64, 64, 10) == 15
     assert L.lot_workspace_bytes(1, 16, 16384, 64, 300, lot.LOT_BF16) == 0      # r too large
     assert L.lot_workspace_bytes(1, 16, 16384, 60, 64, lot.LOT_BF16) == 0       # d % 8 != 0
     assert L.lot_sinkhorn_workspace_bytes(2, 3, 100, 16) > 0
