@@ -1,7 +1,7 @@
 // Thin wrappers over the sm_100a instructions the fused kernels use: mbarrier, TMA tensor
 // loads (no multicast), tcgen05 tensor-core MMA with TMEM accumulators, TMEM loads.
-// Every wait is bounded: it gives up after kSpinLimit polls, raises the CTA's abort flag and
-// the caller-visible LOT_DEV_TIMEOUT status bit, and returns false.
+// Every wait is bounded: it gives up after about kWaitLimitNs of wall time, raises the CTA's
+// abort flag and the caller-visible LOT_DEV_TIMEOUT status bit, and returns false.
 #pragma once
 
 #include <cuda.h>
@@ -11,7 +11,14 @@
 namespace lot {
 namespace sm100 {
 
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint64_t kWaitLimitNs = 1000000000ull;   // one second
+
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
@@ -43,9 +50,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait.  `abort_flag` lives in shared memory; `status` is the global status word.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 1023u) == 1023u && *abort_flag) return false;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
+        }
     }
     *abort_flag = 1;
     atomicOr(status, 4 /* LOT_DEV_TIMEOUT */);
