@@ -110,6 +110,40 @@ LOT_API int lot_sinkhorn(const float *cost, const float *beta, const int32_t *le
                  float *g, float *f, float *plan,
                  void *ws, size_t ws_bytes, lot_stream_t stream);
 
+/*
+ * lot_sinkhorn_static -- lot_sinkhorn for callers that must not allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of the same solve.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a framework whose
+ * allocator owns all device memory and forbids raw allocations, in a real-time or
+ * latency-critical loop where an allocation (which may synchronise the device) is not
+ * acceptable, or in a plug-in that is handed tensors but no allocator.  Such callers cannot
+ * produce the workspace lot_sinkhorn asks for.
+ *
+ * Here the scratch is a fixed array of LOT_STATIC_SCRATCH_BYTES that lives inside the library
+ * image: every device that loads liblot holds that much memory until the process exits,
+ * whether or not this function is ever called.  The call itself allocates nothing and calls
+ * no allocating routine; the caller still provides every input and output buffer.
+ *
+ *   Arguments cost, beta, len, B, H, n, r, eps, iters, g, f, plan, stream: as lot_sinkhorn.
+ *   status_out: device int32 or NULL; receives the device status word of this call.
+ *
+ * Limits and rules
+ *   - lot_sinkhorn_workspace_bytes(B,H,n,r) must not exceed LOT_STATIC_SCRATCH_BYTES;
+ *     larger problems return LOT_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the device address of the array (with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which still holds what the previous call
+ *     left; the part that must start at zero is cleared at the start of every call.  Two
+ *     calls whose work overlaps on the GPU (different streams, no ordering) race on it and
+ *     give undefined results: order them.
+ */
+#define LOT_STATIC_SCRATCH_BYTES (4u << 20)
+LOT_API int lot_sinkhorn_static(const float *cost, const float *beta, const int32_t *len,
+                        int B, int H, int n, int r, float eps, int iters,
+                        float *g, float *f, float *plan, int32_t *status_out,
+                        lot_stream_t stream);
+
 /* Scratch bytes lot_attention_fwd_ex needs for these sizes. */
 LOT_API size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype);
 

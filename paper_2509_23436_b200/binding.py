@@ -29,6 +29,7 @@ SIGNATURES = {
     "lot_cost": (_i, [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp]),
     "lot_sinkhorn_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "lot_sinkhorn": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "lot_sinkhorn_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _vp]),
     "lot_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
     "lot_launch_count": (_i, [_i, _i, _i, _i]),
     "lot_attention_fwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
@@ -124,6 +125,22 @@ def lot_sinkhorn(cost, beta, length, eps, iters, *, want_f=False, want_plan=Fals
                             _dev(ws, "ws"), ws.numel(), _stream(stream))
     _check(st, "lot_sinkhorn")
     return g, f, plan, ws
+
+
+LOT_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def lot_sinkhorn_static(cost, beta, length, eps, iters, g, f=None, plan=None, status_out=None, stream=None):
+    """lot_sinkhorn on the library's built-in scratch array: allocates nothing, so every output
+    (g, and f / plan / status_out if wanted) is a tensor the caller passes in.  Returns g."""
+    B, H, n, r = cost.shape
+    st = lib().lot_sinkhorn_static(_dev(cost, "cost", torch.float32), _dev(beta, "beta", torch.float32),
+                                   _dev(length, "len", torch.int32), B, H, n, r, float(eps), int(iters),
+                                   _dev(g, "g", torch.float32), _dev(f, "f", torch.float32),
+                                   _dev(plan, "plan", torch.float32), _dev(status_out, "status_out", torch.int32),
+                                   _stream(stream))
+    _check(st, "lot_sinkhorn_static")
+    return g
 
 
 def lot_workspace_bytes(B, H, n, d, r, dtype_code) -> int:

@@ -96,6 +96,12 @@ struct Managed {
 Managed g_managed[kMaxDevices];
 std::mutex g_managed_mu;
 
+// Scratch of lot_sinkhorn_static: part of the library image, present on every device that loads
+// it.  In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[LOT_STATIC_SCRATCH_BYTES];
+void *g_static_ptr[kMaxDevices];   // device address of the array, per device (looked up once)
+std::mutex g_static_mu;
+
 } // namespace
 
 extern "C" {
@@ -108,7 +114,7 @@ const char *lot_status_string(int status)
     case LOT_OK: return "LOT_OK";
     case LOT_ERR_INVALID_ARG: return "LOT_ERR_INVALID_ARG: null or misaligned pointer, eps <= 0, iters < 0 or unknown dtype";
     case LOT_ERR_UNSUPPORTED_SHAPE: return "LOT_ERR_UNSUPPORTED_SHAPE: need 1 <= r <= 256, 8 <= d <= 256, d % 8 == 0, B*H <= 32767, n*r and n*d < 2^31";
-    case LOT_ERR_WORKSPACE: return "LOT_ERR_WORKSPACE: workspace null, not 256-byte aligned or too small";
+    case LOT_ERR_WORKSPACE: return "LOT_ERR_WORKSPACE: workspace null, not 256-byte aligned or too small (lot_sinkhorn_static: the problem needs more than LOT_STATIC_SCRATCH_BYTES)";
     case LOT_ERR_CUDA: return "LOT_ERR_CUDA: a CUDA runtime call or kernel launch failed";
     default: return "unknown lot status";
     }
@@ -167,6 +173,39 @@ int lot_sinkhorn(const float *cost, const float *beta, const int32_t *len,
     for (int it = 0; it < iters; ++it)
         if (launch_sinkhorn_pass(a, false, s) != cudaSuccess) return LOT_ERR_CUDA;
     if (launch_sinkhorn_pass(a, true, s) != cudaSuccess) return LOT_ERR_CUDA;
+    return LOT_OK;
+}
+
+int lot_sinkhorn_static(const float *cost, const float *beta, const int32_t *len,
+                        int B, int H, int n, int r, float eps, int iters,
+                        float *g, float *f, float *plan, int32_t *status_out,
+                        lot_stream_t stream)
+{
+    int st = check_dims(B, H, n, r);
+    if (st != LOT_OK) return st;
+    if (status_out && (reinterpret_cast<uintptr_t>(status_out) & 3u)) return LOT_ERR_INVALID_ARG;
+    if (B == 0 || n == 0) return LOT_OK;
+    if (sink_layout(B * H, n, r, 0, 8).total > (size_t)LOT_STATIC_SCRATCH_BYTES) return LOT_ERR_WORKSPACE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LOT_ERR_CUDA;
+    void *ws = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (g_static_ptr[dev] == nullptr) {
+            void *p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+                (void)cudaGetLastError();
+                return LOT_ERR_CUDA;
+            }
+            g_static_ptr[dev] = p;
+        }
+        ws = g_static_ptr[dev];
+    }
+    st = lot_sinkhorn(cost, beta, len, B, H, n, r, eps, iters, g, f, plan, ws, LOT_STATIC_SCRATCH_BYTES, stream);
+    if (st != LOT_OK) return st;
+    if (status_out && cudaMemcpyAsync(status_out, ws, sizeof(int32_t), cudaMemcpyDeviceToDevice,
+                                      (cudaStream_t)stream) != cudaSuccess)
+        return LOT_ERR_CUDA;
     return LOT_OK;
 }
 
