@@ -1,21 +1,30 @@
-// Fused tensor-core path of the LOT attention forward for bf16 tensors (sm_100a).
+// Fused tensor-core path of the LOT attention forward for bf16 tensors (sm_100a): ONE persistent,
+// cooperatively launched kernel runs every Sinkhorn pass and both apply stages.
 //
 // The similarity matrices are never stored: every pass recomputes the logits of a 128-token
 // tile with tcgen05.mma (bf16 tokens x pivots pre-scaled by log2(e)/eps and split into bf16
-// hi + lo parts, f32 accumulation in TMEM), tokens staged by TMA.  One thread owns one token
-// row of the TMEM accumulator, so the row log-sum-exp over the pivots (token update of the
-// Sinkhorn iteration, Eq. (1)-(2) in scaling form) needs no cross-thread traffic, and the
-// column sums over tokens (pivot update) are accumulated per thread over all tiles of a
-// segment and reduced across threads once per segment.
+// hi + lo parts, f32 accumulation in TMEM), tokens staged by TMA.  With the token potential
+// eliminated the state of a solve (Eq. (1)-(2), scaling form) is the pivot potential G:
+//   token update : row log-sum-exp over the pivots (inside a thread quad / a thread)
+//   pivot update : column sums over the tokens of the row-normalised tile, per (slice, side)
 //
-// One launch per pass ("round"); a CTA owns a fixed range of tiles of both sides, split into
-// segments = (slice, side).  Cross-CTA reductions are per-CTA partials merged in slot order by
-// the last CTA to arrive on a ticket (no CTA ever waits for another).
-//   SUM  rounds: both sides, one pivot update of G per round and (slice, side).
-//   WRED round : key side, closing token update, W = Gamma2 V on tensor cores, W' = W / beta.
-//   OUT  round : query side, closing token update, out = softmax-rows x W' on tensor cores.
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 two epilogue
-// groups of 128 threads (group g takes the tiles of parity g and TMEM accumulator g).
+// Work split.  CTA c owns tiles [c*q, (c+1)*q) of the slice-major tile list, for both sides, in
+// every pass; a (slice, side) range of it is a segment.  Pass order: T SUM passes (both sides,
+// one pivot update each), one spare SUM pass for segments that had to repeat an update with
+// (kappa, S) column pairs, the WRED pass (key side: closing token update, W = Gamma2 V on
+// tensor cores, W' = W / beta) and the OUT pass (query side: closing token update,
+// out = softmax-rows x W' on tensor cores).
+//
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-17 four epilogue
+// groups of 128 threads (tile k goes to group k % 4 and TMEM accumulator k % 4).  Producer and
+// MMA issuer never depend on G, so they run ahead across pass boundaries; only an epilogue
+// group waits, per segment, for the potential of that attempt.
+//
+// Cross-CTA protocol (all CTAs are co-resident: cooperative launch, one CTA per SM).  Every
+// group writes its column partial of a segment to its own slot and takes a ticket; the last
+// group to arrive merges all slots in slot order (deterministic), updates G and publishes
+// epoch = attempt + 1 with release semantics; waiters poll epoch with acquire loads.  Every
+// wait, on an mbarrier or on global memory, is bounded in time and raises LOT_DEV_TIMEOUT.
 #include "lot_common.cuh"
 #include "lot_internal.h"
 #include "lot_sm100.cuh"
@@ -28,28 +37,32 @@ namespace fused {
 
 using namespace sm100;
 
-constexpr int kModeSum = 0, kModeWred = 1, kModeOut = 2;
-constexpr int kThreads = 320;
-constexpr int kEpiThreads = 256;
+constexpr int kPhaseSum = 0, kPhaseWred = 1, kPhaseOut = 2;
+constexpr int kGroups = 4;
+constexpr int kEpiThreads = kGroups * 128;
+constexpr int kThreads = 64 + kEpiThreads;
 constexpr int kTileRows = 128;
-constexpr int kPanelBytes = 128 * 128;   // 128 rows x 64 bf16 (one 128-byte-swizzled panel)
-constexpr float kPlainFloor = 8.2718061e-25f;   // 2^-80: smallest column mass the plain sums may report
+constexpr int kDK = 64;                          // head dimension of this path
+constexpr int kStageBytes = kTileRows * kDK * 2; // one token tile: 128 rows x 64 bf16, 128-byte swizzled
+constexpr int kStages = 6;
+constexpr float kPlainFloor = 8.2718061e-25f;    // 2^-80: smallest column mass the plain sums may report
 
 struct alignas(64) FusedParams {
-    CUtensorMap tmQ, tmK, tmV;   // [BH][n][d] bf16, box 64 x 128 x 1
-    CUtensorMap tmZ;             // [2H][RP][d] bf16 (hi, lo of scaled pivots), box 64 x RP x 1
-    CUtensorMap tmW;             // [2BH][d][64] bf16 (hi, lo of W'^T), box 64 x d x 1
+    CUtensorMap tmQ, tmK, tmV;   // [BH][n][64] bf16, box 64 x 128 x 1
+    CUtensorMap tmZ;             // [2H][RP][64] bf16 (hi, lo of scaled pivots), box 64 x RP x 1
     const float *beta;           // [H][r]
     const int32_t *key_len;      // [B] or nullptr
     float *G;                    // [2][BH][RP] pivot potentials, base-2 units (side 0 = queries, 1 = keys)
-    float *part;                 // [2][BH][maxslots][RP][2] column pairs per CTA slot
+    float *part;                 // [2][BH][maxslots*4][RP][2] column pairs per (CTA slot, group)
     unsigned *ticket;            // [2][BH]
+    int *epoch;                  // [2][BH] attempts finished
     int *iter;                   // [2][BH] pivot updates done
-    int *robust;                 // [2][BH] 1 = column sums carried as (kappa, S) pairs
-    float *wpart;                // [BH][maxslots][128][d] per-slot W accumulators (rows 0-63 hi, 64-127 lo)
-    __nv_bfloat16 *Wb;           // [BH][2][d][64] W'^T split hi/lo, pivot-contiguous
+    int *robust;                 // [2][BH] 1 = column sums carried as (kappa, S) pairs (sticky)
+    float *wpart;                // [BH][maxslots][128][64] per-slot W accumulators (rows 0-63 hi, 64-127 lo)
+    __nv_bfloat16 *Wb;           // [BH][2][64][64] W'^T split hi/lo, pivot-contiguous
     unsigned *wticket;           // [BH]
-    __nv_bfloat16 *out;          // [BH][n][d]
+    int *wdone;                  // [BH] 1 = Wb of the slice is final
+    __nv_bfloat16 *out;          // [BH][n][64]
     float *g_nat;                // [2][BH][r] final potentials, natural-log units
     int *status;
     int B, H, n, r, T;
@@ -60,33 +73,38 @@ struct alignas(64) FusedParams {
 };
 
 // ---------------------------------------------------------------------------------------
-// Segment enumeration: identical in every warp role of a CTA.
+// Schedule: the same enumeration in every warp role of a CTA (it depends on launch constants
+// and key_len only).
 // ---------------------------------------------------------------------------------------
 struct Seg {
-    int s, side, b, h, nvalid, t0, t1, slot, nslots, robust, iter;
+    int phase, attempt, extra, s, side, b, h, nvalid, t0, t1, slot, nslots;
 };
 
-template <int MODE>
-struct SegIter {
+struct Sched {
     const FusedParams &P;
-    int u0, u1, s, s_end, side_idx;
-    __device__ explicit SegIter(const FusedParams &p) : P(p)
+    int u0, u1, s_lo, s_hi, pass, s, side_idx;
+    __device__ explicit Sched(const FusedParams &p) : P(p)
     {
         const int NT = p.B * p.H * p.TPS;
         u0 = blockIdx.x * p.q;
         u1 = min(NT, u0 + p.q);
-        s = u0 / p.TPS;
-        s_end = (u1 - 1) / p.TPS;
+        s_lo = u0 / p.TPS;
+        s_hi = (u1 - 1) / p.TPS;
+        pass = p.T == 0 ? 1 : 0;       // passes 0..T-1 SUM, T spare SUM, T+1 WRED, T+2 OUT
+        s = s_lo;
         side_idx = 0;
     }
     __device__ bool next(Seg &g)
     {
-        constexpr int nsides = MODE == kModeSum ? 2 : 1;
-        const int BH = P.B * P.H;
-        while (s <= s_end) {
+        for (;;) {
+            if (pass > P.T + 2) return false;
+            if (s > s_hi) { s = s_lo; side_idx = 0; ++pass; continue; }
+            const int phase = pass <= P.T ? kPhaseSum : (pass == P.T + 1 ? kPhaseWred : kPhaseOut);
+            const int nsides = phase == kPhaseSum ? 2 : 1;
             if (side_idx >= nsides) { side_idx = 0; ++s; continue; }
-            const int side = MODE == kModeSum ? (side_idx == 0 ? 1 : 0) : (MODE == kModeWred ? 1 : 0);
+            const int side = phase == kPhaseSum ? (side_idx == 0 ? 1 : 0) : (phase == kPhaseWred ? 1 : 0);
             ++side_idx;
+            g.phase = phase; g.attempt = pass; g.extra = (phase == kPhaseSum && pass == P.T);
             g.s = s; g.side = side; g.b = s / P.H; g.h = s % P.H;
             g.nvalid = P.n;
             if (side == 1 && P.key_len != nullptr) g.nvalid = min(max(__ldg(P.key_len + g.b), 0), P.n);
@@ -94,142 +112,135 @@ struct SegIter {
             g.t0 = max(u0 - s * P.TPS, 0);
             g.t1 = min(u1 - s * P.TPS, vt);
             if (g.t0 >= g.t1) continue;
-            g.robust = 0; g.iter = 0;
-            if (MODE == kModeSum) {
-                g.iter = __ldcg(P.iter + side * BH + s);
-                if (g.iter >= P.T) continue;
-                g.robust = __ldcg(P.robust + side * BH + s);
-            }
             const int c_lo = (s * P.TPS) / P.q, c_hi = (s * P.TPS + vt - 1) / P.q;
             g.slot = (int)blockIdx.x - c_lo;
             g.nslots = c_hi - c_lo + 1;
             return true;
         }
-        return false;
     }
 };
 
 // ---------------------------------------------------------------------------------------
 // Shared-memory plan
 // ---------------------------------------------------------------------------------------
-template <int DK, int MODE>
 struct Plan {
-    static constexpr int KB = DK / 64;                        // 64-column panels per token tile
-    static constexpr int XS = MODE == kModeSum ? (DK == 64 ? 4 : 3) : (DK == 64 ? 3 : 2);
-    static constexpr int XBYTES = KB * kPanelBytes;
-    static constexpr int ZBYTES = 2 * KB * (64 * 128);        // hi, lo x panels of <= 64 pivot rows
-    static constexpr int VS = MODE == kModeWred ? (DK == 64 ? 3 : 2) : 0;
-    static constexpr int PBUFS = MODE == kModeSum ? 0 : (MODE == kModeWred && DK == 128 ? 1 : 2);
-    static constexpr int PBYTES = MODE == kModeWred ? 2 * kPanelBytes : kPanelBytes;
-    static constexpr int WBYTES = MODE == kModeOut ? 2 * DK * 128 : 0;
+    static constexpr int ZBYTES = 2 * (64 * 128);              // hi, lo panels of <= 64 pivot rows
+    static constexpr int PBYTES = 2 * kStageBytes;             // plan tile as MMA operand: hi and lo panels
+    static constexpr int WBYTES = 2 * kDK * 128;               // W'^T hi, lo
     static constexpr int offX = 0;
-    static constexpr int offZ = offX + XS * XBYTES;
-    static constexpr int offV = offZ + ZBYTES;
-    static constexpr int offP = offV + VS * XBYTES;
-    static constexpr int offW = offP + PBUFS * PBYTES;
-    static constexpr int offBar = offW + WBYTES;              // 64 mbarriers
-    static constexpr int offMisc = offBar + 64 * 8;
-    static constexpr int offG = offMisc + 64;                 // float sG[2][64]
-    static constexpr int offRed = offG + 2 * 64 * 4;          // float sRed[8][64][2]
-    static constexpr int offKap = offRed + 8 * 64 * 2 * 4;    // float sKap[64][256]: per-thread exponents of the
-    static constexpr int total = offKap + (MODE == kModeSum ? 64 * 256 * 4 : 0);   // robust (kappa, S) pairs
-    static constexpr int dyn_bytes = total + 1024;            // slack for 1024-byte alignment
-    static constexpr int tmem_cols = MODE == kModeSum ? 128 : (MODE == kModeWred ? 256 : (DK == 64 ? 256 : 512));
-    static constexpr int colW = 128;                          // first TMEM column of the apply accumulators
+    static constexpr int offZ = offX + kStages * kStageBytes;  // two pivot buffers
+    static constexpr int offP = offZ + 2 * ZBYTES;             // two plan buffers
+    static constexpr int offW = offP + 2 * PBYTES;
+    static constexpr int offBar = offW + WBYTES;               // 64 mbarriers
+    static constexpr int offMisc = offBar + 64 * 8;            // abort flag, TMEM base, flags
+    static constexpr int offG = offMisc + 128;                 // float sG[4][64]
+    static constexpr int offRed = offG + kGroups * 64 * 4;     // float sRed[4][4][64][2]
+    static constexpr int total = offRed + kGroups * 4 * 64 * 2 * 4;
+    static constexpr int dyn_bytes = total + 1024;             // slack for 1024-byte alignment
+    static constexpr int tmem_cols = 512;
+    static constexpr int colW = 256;                           // W accumulator (WRED): 64 columns
+    static constexpr int colO = 320;                           // two output accumulators (OUT): 2 x 64 columns
 };
 
-enum BarId { bXFull = 0, bXEmpty = 4, bZFull = 8, bZEmpty = 9, bAccFull = 10, bAccEmpty = 12, bVFull = 14, bVEmpty = 18,
-             bPFull = 22, bPEmpty = 24, bOFull = 26, bOEmpty = 28, bWFull = 30, bWEmpty = 31, bWqFull = 32, bWqEmpty = 33,
-             bCount = 34 };
-
-// sum-reduce acc[0..N) over the 32 lanes; afterwards lane L holds, in acc[0..N/32) (N >= 32), the
-// totals of columns L*N/32 + j, or for N = 16 lane L holds column L/2 in acc[0].
-template <int N>
-__device__ __forceinline__ void warp_reduce_cols(float (&acc)[N], int lane)
-{
-    int cnt = N / 2;
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        if (cnt >= 1) {
-            const bool up = (lane & off) != 0;
-#pragma unroll
-            for (int j = 0; j < N / 2; ++j) {
-                if (j < cnt) {
-                    float send = up ? acc[j] : acc[j + cnt];
-                    float keep = up ? acc[j + cnt] : acc[j];
-                    acc[j] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-                }
-            }
-            cnt >>= 1;
-        } else {
-            acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], off);
-        }
-    }
-}
-// the same for (kappa, S) pairs
-template <int N>
-__device__ __forceinline__ void warp_reduce_pairs(float (&kap)[N], float (&S)[N], int lane)
-{
-    int cnt = N / 2;
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        if (cnt >= 1) {
-            const bool up = (lane & off) != 0;
-#pragma unroll
-            for (int j = 0; j < N / 2; ++j) {
-                if (j < cnt) {
-                    float sk = up ? kap[j] : kap[j + cnt], ss = up ? S[j] : S[j + cnt];
-                    float kk = up ? kap[j + cnt] : kap[j], ks = up ? S[j + cnt] : S[j];
-                    float ok = __shfl_xor_sync(0xffffffffu, sk, off), os = __shfl_xor_sync(0xffffffffu, ss, off);
-                    pair_merge(kk, ks, ok, os);
-                    kap[j] = kk; S[j] = ks;
-                }
-            }
-            cnt >>= 1;
-        } else {
-            float ok = __shfl_xor_sync(0xffffffffu, kap[0], off), os = __shfl_xor_sync(0xffffffffu, S[0], off);
-            float kk = kap[0], ks = S[0];
-            pair_merge(kk, ks, ok, os);
-            kap[0] = kk; S[0] = ks;
-        }
-    }
-}
-// column held in slot j of lane `lane` after warp_reduce_*<N>
-template <int N>
-__device__ __forceinline__ int reduced_col(int lane, int j)
-{
-    return N >= 32 ? lane * (N / 32) + j : lane / 2;
-}
+enum BarId { bXFull = 0, bXEmpty = 8, bZFull = 16, bZEmpty = 18, bAccFull = 20, bAccEmpty = 24, bPFull = 28, bPEmpty = 30,
+             bOFull = 32, bOEmpty = 34, bWFull = 36, bWEmpty = 37, bWqFull = 38, bWqEmpty = 39, bCount = 40 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 {
     __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t *>(&t);
 }
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ int ld_acquire(const int *p)
+{
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(int *p, int v)
+{
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// Bounded wait until *p >= want (one thread polls).
+__device__ __forceinline__ bool poll_ge(const int *p, int want, volatile int *abort_flag, int *status)
+{
+    if (*abort_flag) return false;
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (ld_acquire(p) >= want) return true;
+        if ((it & 31u) == 31u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
+        }
+        __nanosleep(32);
+    }
+    *abort_flag = 1;
+    atomicOr(status, 4 /* LOT_DEV_TIMEOUT */);
+    return false;
+}
+
+// Quad-layout TMEM load (16 lanes x RP columns): thread L of the warp gets, in v[rep*4 + k],
+// lane L/4 + 8*(k/2) and column rep*8 + 2*(L%4) + (k%2) of the 16-lane block at taddr.
+template <int RP>
+__device__ __forceinline__ void tmem_ld_quad(uint32_t taddr, float *v)
+{
+    uint32_t *r = reinterpret_cast<uint32_t *>(v);
+    if constexpr (RP == 64) {
+        asm volatile("tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+                     "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                     "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                       "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                       "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                       "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                     : "r"(taddr) : "memory");
+    } else if constexpr (RP == 32) {
+        asm volatile("tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+                     "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                       "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                     : "r"(taddr) : "memory");
+    } else {
+        static_assert(RP == 16, "pivot padding");
+        asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                     : "r"(taddr) : "memory");
+    }
+}
 
 // ---------------------------------------------------------------------------------------
-// The round kernel
+// The kernel
 // ---------------------------------------------------------------------------------------
-template <int DK, int RP, int MODE>
+template <int RP>
 __global__ void __launch_bounds__(kThreads, 1)
-fused_round_kernel(const __grid_constant__ FusedParams P)
+fused_forward_kernel(const __grid_constant__ FusedParams P)
 {
-    using PL = Plan<DK, MODE>;
-    constexpr int KB = PL::KB;
+    using PL = Plan;
+    constexpr int DK = kDK;
+    constexpr int NC = RP / 4;          // columns per thread in the quad layout
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + PL::offBar);
     volatile int *sAbort = reinterpret_cast<volatile int *>(smem + PL::offMisc);
     uint32_t *sTmem = reinterpret_cast<uint32_t *>(smem + PL::offMisc + 4);
-    volatile int *sLast = reinterpret_cast<volatile int *>(smem + PL::offMisc + 8);
-    volatile int *sFail = reinterpret_cast<volatile int *>(smem + PL::offMisc + 12);
+    volatile int *sLastW = reinterpret_cast<volatile int *>(smem + PL::offMisc + 8);
+    volatile int *sLast = reinterpret_cast<volatile int *>(smem + PL::offMisc + 16);   // [4]
+    volatile int *sFail = reinterpret_cast<volatile int *>(smem + PL::offMisc + 32);   // [4]
+    volatile int *sFlag = reinterpret_cast<volatile int *>(smem + PL::offMisc + 48);   // [4] per-group scratch flag
     float *sG = reinterpret_cast<float *>(smem + PL::offG);
     float *sRed = reinterpret_cast<float *>(smem + PL::offRed);
     auto bar = [&](int id) { return smem_u32(bars + id); };
-    // whole-warp wait with a warp-uniform verdict (every lane polls; the warp agrees on the result)
-    auto wwait = [&](uint32_t b, uint32_t parity, volatile int *ab, int *st) {
-        const bool r = mbar_wait(b, parity, ab, st);
+    // whole-warp wait with a warp-uniform verdict
+    auto wwait = [&](uint32_t b, uint32_t parity) {
+        const bool r = mbar_wait(b, parity, sAbort, P.status);
         return __all_sync(0xffffffffu, r) != 0;
     };
 
@@ -237,21 +248,18 @@ fused_round_kernel(const __grid_constant__ FusedParams P)
     const int BH = P.B * P.H;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 4; ++i) { mbar_init(bar(bXFull + i), 1); mbar_init(bar(bXEmpty + i), 1); }
-        mbar_init(bar(bZFull), 1); mbar_init(bar(bZEmpty), 1);
+        for (int i = 0; i < kStages; ++i) { mbar_init(bar(bXFull + i), 1); mbar_init(bar(bXEmpty + i), 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(bAccFull + i), 1); mbar_init(bar(bAccEmpty + i), 4);
+            mbar_init(bar(bZFull + i), 1); mbar_init(bar(bZEmpty + i), 1);
             mbar_init(bar(bPFull + i), 4); mbar_init(bar(bPEmpty + i), 1);
             mbar_init(bar(bOFull + i), 1); mbar_init(bar(bOEmpty + i), 4);
         }
-        for (int i = 0; i < 4; ++i) { mbar_init(bar(bVFull + i), 1); mbar_init(bar(bVEmpty + i), 1); }
-        mbar_init(bar(bWFull), 1); mbar_init(bar(bWEmpty), 8);
-        mbar_init(bar(bWqFull), 1); mbar_init(bar(bWqEmpty), 1);
+        for (int i = 0; i < kGroups; ++i) { mbar_init(bar(bAccFull + i), 1); mbar_init(bar(bAccEmpty + i), 4); }
+        mbar_init(bar(bWFull), 1); mbar_init(bar(bWEmpty), 16);
+        mbar_init(bar(bWqFull), 16); mbar_init(bar(bWqEmpty), 1);
         *sAbort = 0;
         fence_barrier_init();
-        prefetch_tensormap(&P.tmQ); prefetch_tensormap(&P.tmK); prefetch_tensormap(&P.tmZ);
-        if (MODE == kModeWred) prefetch_tensormap(&P.tmV);
-        if (MODE == kModeOut) prefetch_tensormap(&P.tmW);
+        prefetch_tensormap(&P.tmQ); prefetch_tensormap(&P.tmK); prefetch_tensormap(&P.tmZ); prefetch_tensormap(&P.tmV);
     }
     if (warp == 1) { tmem_alloc(smem_u32(sTmem), PL::tmem_cols); tmem_relinquish(); }
     tc_fence_before();
@@ -264,226 +272,411 @@ fused_round_kernel(const __grid_constant__ FusedParams P)
     constexpr uint32_t idesc_o = make_idesc_bf16(128, DK, 0, 0);
 
     if (warp == 0) {
-        // ======================= TMA producer =======================
+        // ======================= TMA producer (one lane) =======================
         if (lane == 0) {
-            SegIter<MODE> it(P);
+            Sched it(P);
             Seg g;
-            int k = 0, zc = 0, prev_h = -1, segc = 0;
+            int kx = 0, ztag[2] = {-1, -1}, zuse[2] = {0, 0};
             bool ok = true;
             while (ok && it.next(g)) {
-                if (g.h != prev_h) {
-                    if (zc > 0) ok = mbar_wait(bar(bZEmpty), (zc - 1) & 1, sAbort, P.status);
+                const int idx = g.side * BH + g.s;
+                if (g.extra) {
+                    ok = poll_ge(P.epoch + idx, P.T, sAbort, P.status);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(bar(bZFull), 2 * KB * RP * 128);
-#pragma unroll
-                    for (int part = 0; part < 2; ++part)
-#pragma unroll
-                        for (int kb = 0; kb < KB; ++kb)
-                            tma_load_3d(sbase + PL::offZ + (part * KB + kb) * (64 * 128), &P.tmZ, bar(bZFull),
-                                        kb * 64, 0, g.h * 2 + part);
-                    ++zc; prev_h = g.h;
+                    if (__ldcg(P.robust + idx) == 0) continue;
                 }
-                if (MODE == kModeOut) {
-                    if (segc > 0) ok = mbar_wait(bar(bWqEmpty), (segc - 1) & 1, sAbort, P.status);
+                const int zs = g.h & 1;
+                if (ztag[zs] != g.h) {
+                    if (zuse[zs] > 0) ok = mbar_wait(bar(bZEmpty + zs), (zuse[zs] - 1) & 1, sAbort, P.status);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(bar(bWqFull), PL::WBYTES);
+                    mbar_arrive_expect_tx(bar(bZFull + zs), 2 * RP * 128);
 #pragma unroll
                     for (int part = 0; part < 2; ++part)
-                        tma_load_3d(sbase + PL::offW + part * (DK * 128), &P.tmW, bar(bWqFull), 0, 0, g.s * 2 + part);
+                        tma_load_3d(sbase + PL::offZ + zs * PL::ZBYTES + part * (64 * 128), &P.tmZ, bar(bZFull + zs),
+                                    0, 0, g.h * 2 + part);
+                    ztag[zs] = g.h; ++zuse[zs];
                 }
                 const CUtensorMap *xm = g.side ? &P.tmK : &P.tmQ;
-                for (int t = g.t0; t < g.t1 && ok; ++t, ++k) {
-                    const int st = k % PL::XS, ph = (k / PL::XS) & 1;
-                    ok = mbar_wait(bar(bXEmpty + st), ph ^ 1, sAbort, P.status);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(bar(bXFull + st), PL::XBYTES);
-#pragma unroll
-                    for (int kb = 0; kb < KB; ++kb)
-                        tma_load_3d(sbase + PL::offX + st * PL::XBYTES + kb * kPanelBytes, xm, bar(bXFull + st),
-                                    kb * 64, t * kTileRows, g.s);
-                    if constexpr (MODE == kModeWred) {
-                        const int vs = k % PL::VS, vph = (k / PL::VS) & 1;
-                        ok = mbar_wait(bar(bVEmpty + vs), vph ^ 1, sAbort, P.status);
+                for (int t = g.t0; t < g.t1 && ok; ++t) {
+                    {
+                        const int st = kx % kStages, ph = (kx / kStages) & 1;
+                        ok = mbar_wait(bar(bXEmpty + st), ph ^ 1, sAbort, P.status);
                         if (!ok) break;
-                        mbar_arrive_expect_tx(bar(bVFull + vs), PL::XBYTES);
-#pragma unroll
-                        for (int kb = 0; kb < KB; ++kb)
-                            tma_load_3d(sbase + PL::offV + vs * PL::XBYTES + kb * kPanelBytes, &P.tmV, bar(bVFull + vs),
-                                        kb * 64, t * kTileRows, g.s);
+                        mbar_arrive_expect_tx(bar(bXFull + st), kStageBytes);
+                        tma_load_3d(sbase + PL::offX + st * kStageBytes, xm, bar(bXFull + st), 0, t * kTileRows, g.s);
+                        ++kx;
+                    }
+                    if (g.phase == kPhaseWred) {
+                        const int st = kx % kStages, ph = (kx / kStages) & 1;
+                        ok = mbar_wait(bar(bXEmpty + st), ph ^ 1, sAbort, P.status);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(bar(bXFull + st), kStageBytes);
+                        tma_load_3d(sbase + PL::offX + st * kStageBytes, &P.tmV, bar(bXFull + st), 0, t * kTileRows, g.s);
+                        ++kx;
                     }
                 }
-                ++segc;
+            }
+            if (!ok) {
+                // give the copies still in flight a bounded time to land before the CTA exits
+                const int first = kx > kStages ? kx - kStages : 0;
+                for (int j = first; j < kx; ++j) {
+                    const uint64_t t0 = global_timer_ns();
+                    while (!mbar_try_wait(bar(bXFull + j % kStages), (j / kStages) & 1))
+                        if (global_timer_ns() - t0 > kWaitLimitNs) break;
+                }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ======================= MMA issuer =======================
-        SegIter<MODE> it(P);
+        Sched it(P);
         Seg g;
-        int k = 0, zc = 0, prev_h = -1, segc = 0;
-        bool ok = true;
-        int pend_k = -1, pend_first = 0;      // tile whose apply MMA is still to be issued
+        int k = 0, kx = 0, ztag[2] = {-1, -1}, zuse[2] = {0, 0}, segw = 0, sego = 0;
+        int ka = 0, ko = 0;                   // tiles of the apply passes / of the OUT pass so far
+        bool ok = true, w_open = false;
+        int pend_k = -1, pend_o = 0, pend_first = 0, pend_vs = 0, pend_phase = 0;   // apply MMA still to be issued
 
-        auto issue_apply = [&](int kk, int first) {
-            const int grp = kk & 1, j = kk >> 1;
-            const int pb = PL::PBUFS == 2 ? grp : 0;
-            const int pj = PL::PBUFS == 2 ? j : kk;
-            if (ok) ok = wwait(bar(bPFull + pb), pj & 1, sAbort, P.status);
-            if constexpr (MODE == kModeWred) {
-                const int vs = kk % PL::VS, vph = (kk / PL::VS) & 1;
-                if (ok) ok = wwait(bar(bVFull + vs), vph, sAbort, P.status);
+        auto issue_apply = [&]() {
+            const int pb = pend_k & 1, pj = pend_k >> 1, ob = pend_o & 1, oj = pend_o >> 1;
+            if (ok) ok = wwait(bar(bPFull + pb), pj & 1);
+            const uint32_t pa = sbase + PL::offP + pb * PL::PBYTES;
+            if (pend_phase == kPhaseWred) {
+                const int vs = pend_vs % kStages, vph = (pend_vs / kStages) & 1;
+                if (ok) ok = wwait(bar(bXFull + vs), vph);
                 tc_fence_after();
                 if (ok && lane == 0) {
-                    const uint32_t pa = sbase + PL::offP + pb * PL::PBYTES;
-                    const uint32_t va = sbase + PL::offV + vs * PL::XBYTES;
+                    const uint32_t va = sbase + PL::offX + vs * kStageBytes;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
-                        uint64_t ad = make_smem_desc(pa + ks * 2048, kPanelBytes, 1024);
-                        uint64_t bd = make_smem_desc(va + ks * 2048, kPanelBytes, 1024);
-                        umma_bf16(tmem_base + PL::colW, ad, bd, idesc_w, (first && ks == 0) ? 0u : 1u);
+                        uint64_t ad = make_smem_desc(pa + ks * 2048, kStageBytes, 1024);
+                        uint64_t bd = make_smem_desc(va + ks * 2048, kStageBytes, 1024);
+                        umma_bf16(tmem_base + PL::colW, ad, bd, idesc_w, (pend_first && ks == 0) ? 0u : 1u);
                     }
                     umma_commit(bar(bPEmpty + pb));
-                    umma_commit(bar(bVEmpty + vs));
+                    umma_commit(bar(bXEmpty + vs));
                 }
             } else {
-                if (ok) ok = wwait(bar(bOEmpty + grp), (j & 1) ^ 1, sAbort, P.status);
+                if (ok) ok = wwait(bar(bOEmpty + ob), (oj & 1) ^ 1);
                 tc_fence_after();
                 if (ok && lane == 0) {
-                    const uint32_t pa = sbase + PL::offP + pb * PL::PBYTES;
 #pragma unroll
                     for (int part = 0; part < 2; ++part)
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) {
                             uint64_t ad = make_smem_desc(pa + ks * 32, 16, 1024);
                             uint64_t bd = make_smem_desc(sbase + PL::offW + part * (DK * 128) + ks * 32, 16, 1024);
-                            umma_bf16(tmem_base + PL::colW + grp * DK, ad, bd, idesc_o, (part | ks) ? 1u : 0u);
+                            umma_bf16(tmem_base + PL::colO + ob * DK, ad, bd, idesc_o, (part | ks) ? 1u : 0u);
                         }
                     umma_commit(bar(bPEmpty + pb));
-                    umma_commit(bar(bOFull + grp));
+                    umma_commit(bar(bOFull + ob));
                 }
             }
             __syncwarp();
+            pend_k = -1;
         };
 
         while (ok && it.next(g)) {
-            if (MODE != kModeSum && pend_k >= 0) { issue_apply(pend_k, pend_first); pend_k = -1; }
-            if (MODE == kModeWred && segc > 0) {
-                if (lane == 0) umma_commit(bar(bWFull));                      // W of the previous segment complete
-                if (ok) ok = wwait(bar(bWEmpty), (segc - 1) & 1, sAbort, P.status);
+            const int idx = g.side * BH + g.s;
+            if (g.extra) {
+                int go = 0;
+                if (lane == 0) go = poll_ge(P.epoch + idx, P.T, sAbort, P.status) ? (__ldcg(P.robust + idx) ? 2 : 1) : 0;
+                go = __shfl_sync(0xffffffffu, go, 0);
+                if (go == 0) { ok = false; break; }
+                if (go == 1) continue;
             }
-            if (g.h != prev_h) {
-                if (zc > 0 && lane == 0) umma_commit(bar(bZEmpty));
-                if (ok) ok = wwait(bar(bZFull), zc & 1, sAbort, P.status);
-                ++zc; prev_h = g.h;
+            if (pend_k >= 0) issue_apply();
+            if (w_open) {                                                    // W of the previous WRED segment complete
+                if (ok && lane == 0) umma_commit(bar(bWFull));
+                __syncwarp();
+                w_open = false;
             }
-            if (MODE == kModeOut) {
-                if (segc > 0 && lane == 0) umma_commit(bar(bWqEmpty));
-                if (ok) ok = wwait(bar(bWqFull), segc & 1, sAbort, P.status);
+            if (g.phase == kPhaseWred) {
+                if (segw > 0 && ok) ok = wwait(bar(bWEmpty), (segw - 1) & 1);
+                ++segw;
+                w_open = true;
+            }
+            const int zs = g.h & 1;
+            if (ztag[zs] != g.h) {
+                if (zuse[zs] > 0 && lane == 0) umma_commit(bar(bZEmpty + zs));
+                __syncwarp();
+                if (ok) ok = wwait(bar(bZFull + zs), zuse[zs] & 1);
+                ztag[zs] = g.h; ++zuse[zs];
+            }
+            if (g.phase == kPhaseOut) {
+                if (sego > 0 && lane == 0) umma_commit(bar(bWqEmpty));
+                __syncwarp();
+                if (ok) ok = wwait(bar(bWqFull), sego & 1);
+                ++sego;
             }
             for (int t = g.t0; t < g.t1 && ok; ++t, ++k) {
-                const int grp = k & 1, j = k >> 1;
-                const int st = k % PL::XS, ph = (k / PL::XS) & 1;
-                ok = wwait(bar(bXFull + st), ph, sAbort, P.status);
-                if (ok) ok = wwait(bar(bAccEmpty + grp), (j & 1) ^ 1, sAbort, P.status);
+                const int grp = k & 3, j = k >> 2;
+                const int st = kx % kStages, ph = (kx / kStages) & 1;
+                ok = wwait(bar(bXFull + st), ph);
+                if (ok) ok = wwait(bar(bAccEmpty + grp), (j & 1) ^ 1);
                 tc_fence_after();
                 if (ok && lane == 0) {
-                    const uint32_t xa = sbase + PL::offX + st * PL::XBYTES;
+                    const uint32_t xa = sbase + PL::offX + st * kStageBytes;
+                    const uint32_t za = sbase + PL::offZ + zs * PL::ZBYTES;
 #pragma unroll
                     for (int part = 0; part < 2; ++part)
 #pragma unroll
                         for (int kk = 0; kk < DK / 16; ++kk) {
-                            const int kb = kk / 4, ko = (kk % 4) * 32;
-                            uint64_t ad = make_smem_desc(xa + kb * kPanelBytes + ko, 16, 1024);
-                            uint64_t bd = make_smem_desc(sbase + PL::offZ + (part * KB + kb) * (64 * 128) + ko, 16, 1024);
+                            uint64_t ad = make_smem_desc(xa + kk * 32, 16, 1024);
+                            uint64_t bd = make_smem_desc(za + part * (64 * 128) + kk * 32, 16, 1024);
                             umma_bf16(tmem_base + grp * RP, ad, bd, idesc_cost, (part | kk) ? 1u : 0u);
                         }
                     umma_commit(bar(bXEmpty + st));
                     umma_commit(bar(bAccFull + grp));
                 }
                 __syncwarp();
-                if (MODE != kModeSum) {
-                    if (pend_k >= 0) issue_apply(pend_k, pend_first);
-                    pend_k = k; pend_first = (t == g.t0);
+                ++kx;
+                if (g.phase != kPhaseSum) {
+                    const int vs = kx;
+                    if (g.phase == kPhaseWred) ++kx;      // the value tile sits in the next ring stage
+                    if (pend_k >= 0) issue_apply();
+                    pend_k = ka++; pend_first = (t == g.t0); pend_vs = vs; pend_phase = g.phase;
+                    if (g.phase == kPhaseOut) pend_o = ko++;
                 }
             }
-            ++segc;
         }
-        if (MODE != kModeSum && pend_k >= 0 && ok) { issue_apply(pend_k, pend_first); pend_k = -1; }
-        if (MODE == kModeWred && segc > 0 && ok && lane == 0) umma_commit(bar(bWFull));
+        if (pend_k >= 0 && ok) issue_apply();
+        if (w_open && ok && lane == 0) umma_commit(bar(bWFull));
         __syncwarp();
     } else {
-        // ======================= epilogue (8 warps) =======================
-        const int ew = warp - 2, grp = ew >> 2, qd = warp & 3;
-        const int etid = threadIdx.x - 64, gtid = etid & 127;
-        const int rit = qd * 32 + lane;                                   // row inside the tile = TMEM lane
+        // ======================= epilogue (16 warps, 4 groups) =======================
+        const int ew = warp - 2, grp = ew >> 2, w4 = ew & 3, qd = warp & 3;
+        const int etid = threadIdx.x - 64, gtid = w4 * 32 + lane;
+        const int rq = lane >> 2, cq = lane & 3;                          // quad layout: row and column quarter
+        const int rit = qd * 32 + lane;                                   // row-per-thread layout: row inside the tile
         const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
         float *myG = sG + grp * 64;
-        SegIter<MODE> it(P);
+        float *myRed = sRed + grp * (4 * 64 * 2);
+        Sched it(P);
         Seg g;
-        int k = 0, segc = 0;
+        int k = 0, ka = 0, ko = 0, segw = 0, sego = 0;
         bool ok = true;
 
-        float acc[RP];      // plain column sums, or S of the (kappa, S) pairs
-        float *myKap = reinterpret_cast<float *>(smem + PL::offKap) + etid;   // kappa of column c at myKap[c * 256]
-
         while (it.next(g)) {
+            const int idx = g.side * BH + g.s;
+            // ---- wait until the potential this segment needs is published
+            if (gtid == 0) {
+                bool w = true;
+                if (g.phase == kPhaseSum) w = poll_ge(P.epoch + idx, g.attempt, sAbort, P.status);
+                else {
+                    w = poll_ge(P.iter + idx, P.T, sAbort, P.status);
+                    if (g.phase == kPhaseOut) {
+                        int kv = P.n;
+                        if (P.key_len != nullptr) kv = min(max(__ldg(P.key_len + g.b), 0), P.n);
+                        if (w && kv > 0) w = poll_ge(P.wdone + g.s, 1, sAbort, P.status);
+                    }
+                }
+                sFlag[grp] = (g.extra && w) ? __ldcg(P.robust + idx) : 1;
+            }
             named_bar_sync(1 + grp, 128);
-            if (gtid < RP) myG[gtid] = gtid < P.r ? __ldcg(P.G + ((size_t)g.side * BH + g.s) * RP + gtid) : neg_inf();
+            if (*sAbort) ok = false;
+            const int go = sFlag[grp];
+            const int rb = g.phase == kPhaseSum ? __ldcg(P.robust + idx) : 0;
             named_bar_sync(1 + grp, 128);
+            if (g.extra && go == 0) continue;                           // this segment needed no repeat
+
+            if (g.phase == kPhaseSum) {
+                // ================= SUM: quad layout, column sums in registers =================
+                float Gr[NC], acc[NC], kap[NC];
 #pragma unroll
-            for (int c = 0; c < RP; ++c) acc[c] = 0.f;
-            if (MODE == kModeSum && g.robust) {
+                for (int ci = 0; ci < NC; ++ci) {
+                    const int col = (ci >> 1) * 8 + 2 * cq + (ci & 1);
+                    Gr[ci] = col < P.r ? __ldcg(P.G + (size_t)idx * RP + col) : neg_inf();
+                    acc[ci] = 0.f; kap[ci] = neg_inf();
+                }
+                for (int t = g.t0; t < g.t1; ++t, ++k) {
+                    if ((k & 3) != grp) continue;
+                    const int j = k >> 2;
+                    if (ok) ok = wwait(bar(bAccFull + grp), j & 1);
+                    if (!ok) continue;
+                    tc_fence_after();
 #pragma unroll
-                for (int c = 0; c < RP; ++c) myKap[c * 256] = neg_inf();
+                    for (int half = 0; half < 2; ++half) {
+                        float v[2 * NC];
+                        tmem_ld_quad<RP>(lane_addr + ((uint32_t)(half * 16) << 16) + grp * RP, v);
+                        tmem_wait_ld();
+                        if (half == 1) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar(bAccEmpty + grp));
+                        }
+                        const int rowA = t * kTileRows + qd * 32 + half * 16 + rq, rowB = rowA + 8;
+                        float mA = neg_inf(), mB = neg_inf();
+#pragma unroll
+                        for (int rep = 0; rep < NC / 2; ++rep) {
+                            v[rep * 4 + 0] += Gr[rep * 2]; v[rep * 4 + 1] += Gr[rep * 2 + 1];
+                            v[rep * 4 + 2] += Gr[rep * 2]; v[rep * 4 + 3] += Gr[rep * 2 + 1];
+                            mA = max3(mA, v[rep * 4 + 0], v[rep * 4 + 1]);
+                            mB = max3(mB, v[rep * 4 + 2], v[rep * 4 + 3]);
+                        }
+                        mA = fmaxf(mA, __shfl_xor_sync(0xffffffffu, mA, 1));
+                        mB = fmaxf(mB, __shfl_xor_sync(0xffffffffu, mB, 1));
+                        mA = fmaxf(mA, __shfl_xor_sync(0xffffffffu, mA, 2));
+                        mB = fmaxf(mB, __shfl_xor_sync(0xffffffffu, mB, 2));
+                        float sA0 = 0.f, sA1 = 0.f, sB0 = 0.f, sB1 = 0.f;
+                        if (!rb) {
+#pragma unroll
+                            for (int rep = 0; rep < NC / 2; ++rep) {
+                                v[rep * 4 + 0] = ex2(v[rep * 4 + 0] - mA); sA0 += v[rep * 4 + 0];
+                                v[rep * 4 + 1] = ex2(v[rep * 4 + 1] - mA); sA1 += v[rep * 4 + 1];
+                                v[rep * 4 + 2] = ex2(v[rep * 4 + 2] - mB); sB0 += v[rep * 4 + 2];
+                                v[rep * 4 + 3] = ex2(v[rep * 4 + 3] - mB); sB1 += v[rep * 4 + 3];
+                            }
+                        } else {
+#pragma unroll
+                            for (int rep = 0; rep < NC / 2; ++rep) {
+                                sA0 += ex2(v[rep * 4 + 0] - mA); sA1 += ex2(v[rep * 4 + 1] - mA);
+                                sB0 += ex2(v[rep * 4 + 2] - mB); sB1 += ex2(v[rep * 4 + 3] - mB);
+                            }
+                        }
+                        float sA = sA0 + sA1, sB = sB0 + sB1;
+                        sA += __shfl_xor_sync(0xffffffffu, sA, 1);
+                        sB += __shfl_xor_sync(0xffffffffu, sB, 1);
+                        sA += __shfl_xor_sync(0xffffffffu, sA, 2);
+                        sB += __shfl_xor_sync(0xffffffffu, sB, 2);
+                        if (!rb) {
+                            const float wA = rowA < g.nvalid ? __fdividef(1.f, sA) : 0.f;
+                            const float wB = rowB < g.nvalid ? __fdividef(1.f, sB) : 0.f;
+#pragma unroll
+                            for (int ci = 0; ci < NC; ++ci) {
+                                acc[ci] = fmaf(v[(ci >> 1) * 4 + (ci & 1)], wA, acc[ci]);
+                                acc[ci] = fmaf(v[(ci >> 1) * 4 + 2 + (ci & 1)], wB, acc[ci]);
+                            }
+                        } else {
+                            // exact log2 of every normalised entry, added to (kappa, S) pairs
+                            const float MA = mA + lg2(sA), MB = mB + lg2(sB);
+#pragma unroll
+                            for (int ci = 0; ci < NC; ++ci) {
+                                const int col = (ci >> 1) * 8 + 2 * cq + (ci & 1);
+                                if (col < P.r) {
+                                    if (rowA < g.nvalid) pair_add(kap[ci], acc[ci], v[(ci >> 1) * 4 + (ci & 1)] - MA);
+                                    if (rowB < g.nvalid) pair_add(kap[ci], acc[ci], v[(ci >> 1) * 4 + 2 + (ci & 1)] - MB);
+                                }
+                            }
+                        }
+                    }
+                }
+                // ---- group partial: rows of the warp (lanes with equal cq), then the 4 warps
+#pragma unroll
+                for (int off = 4; off <= 16; off <<= 1) {
+#pragma unroll
+                    for (int ci = 0; ci < NC; ++ci) {
+                        if (rb) {
+                            const float ok2 = __shfl_xor_sync(0xffffffffu, kap[ci], off);
+                            const float os2 = __shfl_xor_sync(0xffffffffu, acc[ci], off);
+                            pair_merge(kap[ci], acc[ci], ok2, os2);
+                        } else {
+                            acc[ci] += __shfl_xor_sync(0xffffffffu, acc[ci], off);
+                        }
+                    }
+                }
+                if (rq == 0) {
+#pragma unroll
+                    for (int ci = 0; ci < NC; ++ci) {
+                        const int col = (ci >> 1) * 8 + 2 * cq + (ci & 1);
+                        myRed[(w4 * 64 + col) * 2] = rb ? kap[ci] : 0.f;
+                        myRed[(w4 * 64 + col) * 2 + 1] = acc[ci];
+                    }
+                }
+                named_bar_sync(1 + grp, 128);
+                if (gtid < RP) {
+                    float kk = myRed[gtid * 2], ss = myRed[gtid * 2 + 1];
+#pragma unroll
+                    for (int w = 1; w < 4; ++w) {
+                        if (rb) pair_merge(kk, ss, myRed[(w * 64 + gtid) * 2], myRed[(w * 64 + gtid) * 2 + 1]);
+                        else ss += myRed[(w * 64 + gtid) * 2 + 1];
+                    }
+                    float *dst = P.part + ((((size_t)idx * P.maxslots + g.slot) * 4 + grp) * RP + gtid) * 2;
+                    __stcg(reinterpret_cast<float2 *>(dst), make_float2(kk, ss));
+                    __threadfence();
+                }
+                named_bar_sync(1 + grp, 128);
+                if (gtid == 0) {
+                    __threadfence();
+                    const unsigned tk = atomicAdd(P.ticket + idx, 1u);
+                    sLast[grp] = (tk == (unsigned)(g.nslots * 4) - 1u);
+                    sFail[grp] = 0;
+                }
+                named_bar_sync(1 + grp, 128);
+                if (sLast[grp]) {
+                    // ---- last group of the (slice, side): merge every slot in slot order, update G
+                    __threadfence();
+                    const int nparts = g.nslots * 4;
+                    const int col = gtid & 63, hsel = gtid >> 6;
+                    float kk = rb ? neg_inf() : 0.f, ss = 0.f;
+                    if (col < RP) {
+                        const float *src = P.part + ((size_t)idx * P.maxslots * 4) * RP * 2 + col * 2;
+                        for (int p = hsel; p < nparts; p += 2) {
+                            const float2 pr = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)p * RP * 2));
+                            if (rb) pair_merge(kk, ss, pr.x, pr.y);
+                            else ss += pr.y;
+                        }
+                    }
+                    if (hsel == 1) { myRed[col * 2] = kk; myRed[col * 2 + 1] = ss; }
+                    named_bar_sync(1 + grp, 128);
+                    if (hsel == 0 && col < P.r) {
+                        if (rb) pair_merge(kk, ss, myRed[col * 2], myRed[col * 2 + 1]);
+                        else ss += myRed[col * 2 + 1];
+                        if (!rb && !(ss >= kPlainFloor && ss <= 3.0e38f)) sFail[grp] = 1;
+                    }
+                    named_bar_sync(1 + grp, 128);
+                    const int fail = sFail[grp];
+                    const int itn = __ldcg(P.iter + idx);
+                    if (!fail && hsel == 0 && col < P.r) {
+                        float *gp = P.G + (size_t)idx * RP + col;
+                        const float gn = __ldcg(gp) + lg2(__ldg(P.beta + g.h * P.r + col) * (float)g.nvalid) - (kk + lg2(ss));
+                        if (!isfinite(gn)) atomicOr(P.status, 1 /* LOT_DEV_NONFINITE */);
+                        __stcg(gp, gn);
+                        if (itn + 1 == P.T) P.g_nat[(size_t)idx * P.r + col] = gn * P.eps_ln2;
+                        __threadfence();
+                    }
+                    named_bar_sync(1 + grp, 128);
+                    if (gtid == 0) {
+                        __stcg(P.ticket + idx, 0u);
+                        if (fail) __stcg(P.robust + idx, 1);
+                        __threadfence();
+                        if (!fail) st_release(P.iter + idx, itn + 1);
+                        st_release(P.epoch + idx, g.attempt + 1);
+                    }
+                }
+                continue;
             }
 
+            // ================= WRED / OUT: one thread per token row =================
+            if (gtid < RP) myG[gtid] = gtid < P.r ? __ldcg(P.G + (size_t)idx * RP + gtid) : neg_inf();
+            if (g.phase == kPhaseOut) {
+                // stage W'^T (hi, lo) of this slice as the B operand: 128-byte rows, 16-byte chunks xor row%8
+                if (sego > 0 && ok) ok = wwait(bar(bWqEmpty), (sego - 1) & 1);
+                const uint4 *src = reinterpret_cast<const uint4 *>(P.Wb + (size_t)g.s * 2 * DK * 64);
+#pragma unroll
+                for (int rep = 0; rep < 2; ++rep) {
+                    const int c = etid + rep * kEpiThreads;          // 1024 chunks of 16 bytes
+                    const int part = c >> 9, row = (c >> 3) & 63, ch = c & 7;
+                    const uint4 val = __ldcg(src + c);
+                    *reinterpret_cast<uint4 *>(smem + PL::offW + part * (DK * 128) + row * 128 + ((ch ^ (row & 7)) * 16)) = val;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(bWqFull));
+                ++sego;
+            }
+            named_bar_sync(1 + grp, 128);
+
             for (int t = g.t0; t < g.t1; ++t, ++k) {
-                if ((k & 1) != grp) continue;
-                const int j = k >> 1;
-                if (ok) ok = wwait(bar(bAccFull + grp), j & 1, sAbort, P.status);
+                const int pb = ka & 1, pj = ka >> 1, ob = ko & 1, oj = ko >> 1;
+                ++ka;
+                if (g.phase == kPhaseOut) ++ko;
+                if ((k & 3) != grp) continue;
+                const int j = k >> 2;
+                if (ok) ok = wwait(bar(bAccFull + grp), j & 1);
                 if (!ok) continue;
                 tc_fence_after();
                 const int row = t * kTileRows + rit;
                 const bool valid = row < g.nvalid;
-                if (MODE == kModeSum && g.robust) {
-                    // ---- robust sums: three sweeps over the accumulator in 16-column chunks
-                    float m = neg_inf();
-#pragma unroll
-                    for (int c0 = 0; c0 < RP; c0 += 16) {
-                        float v[16];
-                        tmem_ld16(lane_addr + grp * RP + c0, v);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) m = fmaxf(m, v[c] + myG[c0 + c]);
-                    }
-                    float s = 0.f;
-#pragma unroll
-                    for (int c0 = 0; c0 < RP; c0 += 16) {
-                        float v[16];
-                        tmem_ld16(lane_addr + grp * RP + c0, v);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) s += ex2(v[c] + myG[c0 + c] - m);
-                    }
-                    const float Mi = m + lg2(s);
-#pragma unroll
-                    for (int c0 = 0; c0 < RP; c0 += 16) {
-                        float v[16];
-                        tmem_ld16(lane_addr + grp * RP + c0, v);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            if (valid && c0 + c < P.r) {
-                                float kk = myKap[(c0 + c) * 256];
-                                pair_add(kk, acc[c0 + c], (v[c] + myG[c0 + c] - m) - (Mi - m));
-                                myKap[(c0 + c) * 256] = kk;
-                            }
-                    }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(bAccEmpty + grp));
-                    continue;
-                }
                 float v[RP];
                 tmem_ld<RP>(lane_addr + grp * RP, v);
                 tmem_wait_ld();
@@ -497,180 +690,111 @@ fused_round_kernel(const __grid_constant__ FusedParams P)
 #pragma unroll
                 for (int c = 0; c < RP; ++c) { v[c] = ex2(v[c] - m); s += v[c]; }
                 const float inv = __fdividef(1.f, s);
-                if (MODE == kModeSum) {
-                    const float w = valid ? inv : 0.f;
+                // ---- write the plan tile as an MMA operand
+                ok = wwait(bar(bPEmpty + pb), (pj & 1) ^ 1);
+                if (!ok) continue;
+                uint8_t *prow = smem + PL::offP + pb * PL::PBYTES + rit * 128;
+                const float w = g.phase == kPhaseWred ? (valid ? inv : 0.f) : 1.f;
 #pragma unroll
-                    for (int c = 0; c < RP; ++c) acc[c] = fmaf(v[c], w, acc[c]);
-                } else {
-                    // ---- write the plan tile as an MMA operand (128-byte rows, 16-byte chunks xor row%8)
-                    const int pb = PL::PBUFS == 2 ? grp : 0;
-                    const int pj = PL::PBUFS == 2 ? j : k;
-                    ok = wwait(bar(bPEmpty + pb), (pj & 1) ^ 1, sAbort, P.status);
-                    if (!ok) continue;
-                    uint8_t *prow = smem + PL::offP + pb * PL::PBYTES + rit * 128;
-                    const float w = MODE == kModeWred ? (valid ? inv : 0.f) : 1.f;
+                for (int c8 = 0; c8 < 8; ++c8) {
+                    uint32_t hi[4], lo[4];
 #pragma unroll
-                    for (int c8 = 0; c8 < 8; ++c8) {
-                        uint32_t hi[4], lo[4];
-#pragma unroll
-                        for (int e2 = 0; e2 < 4; ++e2) {
-                            const int c = c8 * 8 + e2 * 2;
-                            float a0 = c < RP ? v[c < RP ? c : 0] * w : 0.f;
-                            float a1 = c + 1 < RP ? v[c + 1 < RP ? c + 1 : 0] * w : 0.f;
-                            __nv_bfloat162 hh = __floats2bfloat162_rn(a0, a1);
-                            hi[e2] = *reinterpret_cast<uint32_t *>(&hh);
-                            if (MODE == kModeWred) lo[e2] = pack_bf16(a0 - __low2float(hh), a1 - __high2float(hh));
-                        }
-                        const int pc = (c8 ^ (rit & 7)) * 16;
-                        *reinterpret_cast<uint4 *>(prow + pc) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                        if (MODE == kModeWred)
-                            *reinterpret_cast<uint4 *>(prow + kPanelBytes + pc) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    for (int e2 = 0; e2 < 4; ++e2) {
+                        const int c = c8 * 8 + e2 * 2;
+                        const float a0 = c < RP ? v[c < RP ? c : 0] * w : 0.f;
+                        const float a1 = c + 1 < RP ? v[c + 1 < RP ? c + 1 : 0] * w : 0.f;
+                        __nv_bfloat162 hh = __floats2bfloat162_rn(a0, a1);
+                        hi[e2] = *reinterpret_cast<uint32_t *>(&hh);
+                        lo[e2] = pack_bf16(a0 - __low2float(hh), a1 - __high2float(hh));
                     }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(bPFull + pb));
-                    if (MODE == kModeOut) {
-                        ok = wwait(bar(bOFull + grp), j & 1, sAbort, P.status);
-                        if (!ok) continue;
-                        tc_fence_after();
-                        float o[DK];
-                        tmem_ld<DK>(lane_addr + PL::colW + grp * DK, o);
-                        tmem_wait_ld();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(bOEmpty + grp));
-                        if (row < P.n) {
-                            __nv_bfloat16 *orow = P.out + ((size_t)g.s * P.n + row) * DK;
+                    const int pc = (c8 ^ (rit & 7)) * 16;
+                    *reinterpret_cast<uint4 *>(prow + pc) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    if (g.phase == kPhaseWred)
+                        *reinterpret_cast<uint4 *>(prow + kStageBytes + pc) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(bPFull + pb));
+                if (g.phase == kPhaseOut) {
+                    ok = wwait(bar(bOFull + ob), oj & 1);
+                    if (!ok) continue;
+                    tc_fence_after();
+                    __nv_bfloat16 *orow = P.out + ((size_t)g.s * P.n + row) * DK;
 #pragma unroll
-                            for (int c = 0; c < DK; c += 8) {
+                    for (int c0 = 0; c0 < DK; c0 += 32) {
+                        float o[32];
+                        tmem_ld32(lane_addr + PL::colO + ob * DK + c0, o);
+                        tmem_wait_ld();
+                        if (c0 + 32 == DK) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar(bOEmpty + ob));
+                        }
+                        if (row < P.n) {
+#pragma unroll
+                            for (int c = 0; c < 32; c += 8) {
                                 uint4 pk;
                                 pk.x = pack_bf16(o[c] * inv, o[c + 1] * inv);
                                 pk.y = pack_bf16(o[c + 2] * inv, o[c + 3] * inv);
                                 pk.z = pack_bf16(o[c + 4] * inv, o[c + 5] * inv);
                                 pk.w = pack_bf16(o[c + 6] * inv, o[c + 7] * inv);
-                                *reinterpret_cast<uint4 *>(orow + c) = pk;
+                                *reinterpret_cast<uint4 *>(orow + c0 + c) = pk;
                             }
                         }
                     }
                 }
             }
 
-            // ------------------------------ segment end ------------------------------
-            if (MODE == kModeSum) {
-                constexpr int NJ = RP >= 32 ? RP / 32 : 1;
-                if (g.robust) {
-                    // slow path: merge the 32 lanes' pairs column by column
-#pragma unroll
-                    for (int c = 0; c < RP; ++c) {
-                        float kk = myKap[c * 256], ss = acc[c];
-#pragma unroll
-                        for (int off = 16; off >= 1; off >>= 1) {
-                            float ok2 = __shfl_xor_sync(0xffffffffu, kk, off), os2 = __shfl_xor_sync(0xffffffffu, ss, off);
-                            pair_merge(kk, ss, ok2, os2);
-                        }
-                        if (lane == 0) { sRed[(ew * 64 + c) * 2] = kk; sRed[(ew * 64 + c) * 2 + 1] = ss; }
-                    }
-                } else {
-                    warp_reduce_cols<RP>(acc, lane);
-                    if (RP >= 32 || (lane & 1) == 0) {
-#pragma unroll
-                        for (int jx = 0; jx < NJ; ++jx) {
-                            const int col = reduced_col<RP>(lane, jx);
-                            sRed[(ew * 64 + col) * 2] = 0.f;
-                            sRed[(ew * 64 + col) * 2 + 1] = acc[jx];
-                        }
-                    }
-                }
-                named_bar_sync(3, kEpiThreads);
-                if (etid < RP) {
-                    float kk = sRed[etid * 2], ss = sRed[etid * 2 + 1];
-#pragma unroll
-                    for (int w = 1; w < 8; ++w) {
-                        if (g.robust) pair_merge(kk, ss, sRed[(w * 64 + etid) * 2], sRed[(w * 64 + etid) * 2 + 1]);
-                        else ss += sRed[(w * 64 + etid) * 2 + 1];
-                    }
-                    float *dst = P.part + ((((size_t)g.side * BH + g.s) * P.maxslots + g.slot) * RP + etid) * 2;
-                    __stcg(dst, kk);
-                    __stcg(dst + 1, ss);
-                    __threadfence();
-                }
-                named_bar_sync(3, kEpiThreads);
-                if (etid == 0) {
-                    __threadfence();
-                    unsigned tk = atomicAdd(P.ticket + g.side * BH + g.s, 1u);
-                    *sLast = (tk == (unsigned)g.nslots - 1u);
-                    *sFail = 0;
-                }
-                named_bar_sync(3, kEpiThreads);
-                if (*sLast) {
-                    __threadfence();
-                    float kk = g.robust ? neg_inf() : 0.f, ss = 0.f;
-                    if (etid < P.r) {
-                        for (int sl = 0; sl < g.nslots; ++sl) {
-                            const float *src = P.part + ((((size_t)g.side * BH + g.s) * P.maxslots + sl) * RP + etid) * 2;
-                            if (g.robust) pair_merge(kk, ss, __ldcg(src), __ldcg(src + 1));
-                            else ss += __ldcg(src + 1);
-                        }
-                        if (!g.robust && !(ss >= kPlainFloor && ss <= 3.0e38f)) *sFail = 1;
-                    }
-                    named_bar_sync(3, kEpiThreads);
-                    const int fail = *sFail;
-                    if (!fail && etid < P.r) {
-                        float *gp = P.G + ((size_t)g.side * BH + g.s) * RP + etid;
-                        const float gn = *gp + lg2(__ldg(P.beta + g.h * P.r + etid) * (float)g.nvalid) - (kk + lg2(ss));
-                        if (!isfinite(gn)) atomicOr(P.status, 1 /* LOT_DEV_NONFINITE */);
-                        *gp = gn;
-                        if (g.iter + 1 == P.T) P.g_nat[((size_t)g.side * BH + g.s) * P.r + etid] = gn * P.eps_ln2;
-                    }
-                    if (etid == 0) {
-                        if (fail) P.robust[g.side * BH + g.s] = 1;
-                        else P.iter[g.side * BH + g.s] = g.iter + 1;
-                        P.ticket[g.side * BH + g.s] = 0u;
-                    }
-                }
-            } else if (MODE == kModeWred) {
-                // the W accumulator of this segment: every group reads half of the channels of its lanes
-                if (ok) ok = wwait(bar(bWFull), segc & 1, sAbort, P.status);
+            if (g.phase == kPhaseWred) {
+                // ---- W accumulator of this segment: warp (qd, grp) takes its 32 lanes x 16 channels
+                if (ok) ok = wwait(bar(bWFull), segw & 1);
                 if (ok) {
                     tc_fence_after();
-                    float w[DK / 2];
-                    tmem_ld<DK / 2>(lane_addr + PL::colW + grp * (DK / 2), w);
+                    float wv[16];
+                    tmem_ld16(lane_addr + PL::colW + grp * 16, wv);
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(bWEmpty));
-                    float *dst = P.wpart + (((size_t)g.s * P.maxslots + g.slot) * 128 + rit) * DK + grp * (DK / 2);
+                    float *dst = P.wpart + (((size_t)g.s * P.maxslots + g.slot) * 128 + rit) * DK + grp * 16;
 #pragma unroll
-                    for (int c = 0; c < DK / 2; c += 4) __stcg(reinterpret_cast<float4 *>(dst + c), make_float4(w[c], w[c + 1], w[c + 2], w[c + 3]));
+                    for (int c = 0; c < 16; c += 4)
+                        __stcg(reinterpret_cast<float4 *>(dst + c), make_float4(wv[c], wv[c + 1], wv[c + 2], wv[c + 3]));
                     __threadfence();
                 }
-                named_bar_sync(3, kEpiThreads);
+                ++segw;
+                named_bar_sync(5, kEpiThreads);
                 if (etid == 0) {
                     __threadfence();
-                    unsigned tk = atomicAdd(P.wticket + g.s, 1u);
-                    *sLast = (tk == (unsigned)g.nslots - 1u);
+                    const unsigned tk = atomicAdd(P.wticket + g.s, 1u);
+                    *sLastW = (tk == (unsigned)g.nslots - 1u) && !*sAbort;
                 }
-                named_bar_sync(3, kEpiThreads);
-                if (*sLast) {
+                named_bar_sync(5, kEpiThreads);
+                if (*sLastW) {
                     __threadfence();
                     const float mass = g.nvalid > 0 ? 1.f / (float)g.nvalid : 0.f;
-                    for (int idx = etid; idx < 64 * DK; idx += kEpiThreads) {
-                        const int tt = idx / DK, c = idx % DK;
+                    for (int e = etid; e < 64 * DK; e += kEpiThreads) {
+                        const int tt = e / DK, c = e % DK;
                         float sum = 0.f;
                         for (int sl = 0; sl < g.nslots; ++sl) {
                             const float *src = P.wpart + (((size_t)g.s * P.maxslots + sl) * 128) * DK + c;
                             sum += __ldcg(src + (size_t)tt * DK) + __ldcg(src + (size_t)(64 + tt) * DK);
                         }
-                        float wv = tt < P.r ? sum * mass / __ldg(P.beta + g.h * P.r + tt) : 0.f;
-                        __nv_bfloat16 hi = __float2bfloat16_rn(wv);
-                        __nv_bfloat16 lo = __float2bfloat16_rn(wv - __bfloat162float(hi));
+                        const float wv = tt < P.r ? sum * mass / __ldg(P.beta + g.h * P.r + tt) : 0.f;
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(wv);
+                        const __nv_bfloat16 lo = __float2bfloat16_rn(wv - __bfloat162float(hi));
                         P.Wb[(((size_t)g.s * 2 + 0) * DK + c) * 64 + tt] = hi;
                         P.Wb[(((size_t)g.s * 2 + 1) * DK + c) * 64 + tt] = lo;
                     }
-                    if (etid == 0) P.wticket[g.s] = 0u;
+                    __threadfence();
+                    named_bar_sync(5, kEpiThreads);
+                    if (etid == 0) {
+                        __stcg(P.wticket + g.s, 0u);
+                        __threadfence();
+                        st_release(P.wdone + g.s, 1);
+                    }
                 }
             }
-            ++segc;
         }
     }
 
@@ -759,7 +883,7 @@ static inline int pad_r(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
 
 bool fused_supported(int dtype, int d, int r)
 {
-    return dtype == 1 && d == 64 && r >= 1 && r <= 64;
+    return dtype == 1 && d == fused::kDK && r >= 1 && r <= 64;
 }
 
 void fused_geometry(int B, int H, int n, int *q, int *ctas, int *maxslots)
@@ -785,45 +909,35 @@ FusedLayout fused_layout(int B, int H, int n, int d, int r)
     L.status = o; o += 256;
     L.G = o; o += up256((size_t)2 * BH * RP * 4);
     L.ticket = o; o += up256((size_t)2 * BH * 4);
+    L.epoch = o; o += up256((size_t)2 * BH * 4);
     L.iter = o; o += up256((size_t)2 * BH * 4);
     L.robust = o; o += up256((size_t)2 * BH * 4);
     L.wticket = o; o += up256((size_t)BH * 4);
+    L.wdone = o; o += up256((size_t)BH * 4);
     L.gnat = o; o += up256((size_t)2 * BH * r * 4);
     L.Wb = o; o += up256((size_t)BH * 2 * d * 64 * 2);
     L.head_end = o;
     L.zprep = o; o += up256((size_t)H * 2 * RP * d * 2);
-    L.part = o; o += up256((size_t)2 * BH * ms * RP * 2 * 4);
+    L.part = o; o += up256((size_t)2 * BH * ms * 4 * RP * 2 * 4);
     L.wpart = o; o += up256((size_t)BH * ms * 128 * d * 4);
     L.total = o;
     return L;
 }
 
-template <int DK, int RP, int MODE>
-static cudaError_t launch_round(const fused::FusedParams &P, int ctas, cudaStream_t st)
+template <int RP>
+static cudaError_t launch_forward(const fused::FusedParams &P, int ctas, cudaStream_t st)
 {
-    using PL = fused::Plan<DK, MODE>;
     static bool attr_set = false;
-    auto kern = fused::fused_round_kernel<DK, RP, MODE>;
+    auto kern = fused::fused_forward_kernel<RP>;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PL::dyn_bytes);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fused::Plan::dyn_bytes);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    kern<<<ctas, fused::kThreads, PL::dyn_bytes, st>>>(P);
-    return cudaGetLastError();
-}
-
-template <int DK, int RP>
-static cudaError_t run_rounds(const fused::FusedParams &P, int ctas, int iters, cudaStream_t st)
-{
-    cudaError_t e;
-    // iters pivot updates, plus one spare round: a slice whose plain column sums underflowed in its
-    // first round repeats that update with (kappa, S) pairs; every other CTA finds nothing to do.
-    const int sum_rounds = iters > 0 ? iters + 1 : 0;
-    for (int it = 0; it < sum_rounds; ++it)
-        if ((e = launch_round<DK, RP, fused::kModeSum>(P, ctas, st)) != cudaSuccess) return e;
-    if ((e = launch_round<DK, RP, fused::kModeWred>(P, ctas, st)) != cudaSuccess) return e;
-    return launch_round<DK, RP, fused::kModeOut>(P, ctas, st);
+    // cooperative launch: the CTAs wait for one another, so all of them must be resident at once
+    void *args[] = {const_cast<fused::FusedParams *>(&P)};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void *>(kern), dim3(ctas), dim3(fused::kThreads), args,
+                                       fused::Plan::dyn_bytes, st);
 }
 
 cudaError_t fused_attention(const void *q, const void *k, const void *v, const float *z, const float *beta,
@@ -840,19 +954,20 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
     FusedParams P;
     memset(&P, 0, sizeof(P));
     __nv_bfloat16 *zp = reinterpret_cast<__nv_bfloat16 *>(w + L.zprep);
-    P.Wb = reinterpret_cast<__nv_bfloat16 *>(w + L.Wb);
     if (!make_map(&P.tmQ, q, BH, n, d, 128) || !make_map(&P.tmK, k, BH, n, d, 128) ||
-        !make_map(&P.tmV, v, BH, n, d, 128) || !make_map(&P.tmZ, zp, 2 * H, RP, d, RP) ||
-        !make_map(&P.tmW, P.Wb, 2 * BH, d, 64, d))
+        !make_map(&P.tmV, v, BH, n, d, 128) || !make_map(&P.tmZ, zp, 2 * H, RP, d, RP))
         return cudaErrorInvalidValue;
     P.beta = beta; P.key_len = key_len;
     P.G = reinterpret_cast<float *>(w + L.G);
     P.part = reinterpret_cast<float *>(w + L.part);
     P.ticket = reinterpret_cast<unsigned *>(w + L.ticket);
+    P.epoch = reinterpret_cast<int *>(w + L.epoch);
     P.iter = reinterpret_cast<int *>(w + L.iter);
     P.robust = reinterpret_cast<int *>(w + L.robust);
     P.wpart = reinterpret_cast<float *>(w + L.wpart);
+    P.Wb = reinterpret_cast<__nv_bfloat16 *>(w + L.Wb);
     P.wticket = reinterpret_cast<unsigned *>(w + L.wticket);
+    P.wdone = reinterpret_cast<int *>(w + L.wdone);
     P.out = static_cast<__nv_bfloat16 *>(out);
     P.g_nat = reinterpret_cast<float *>(w + L.gnat);
     P.status = reinterpret_cast<int *>(w + L.status);
@@ -867,9 +982,9 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
     zprep_kernel<<<(total + 255) / 256, 256, 0, st>>>(z, zp, key_len, P.status, B, H, r, RP, d, scale);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-    if (RP == 16) e = run_rounds<64, 16>(P, ctas, iters, st);
-    else if (RP == 32) e = run_rounds<64, 32>(P, ctas, iters, st);
-    else e = run_rounds<64, 64>(P, ctas, iters, st);
+    if (RP == 16) e = launch_forward<16>(P, ctas, st);
+    else if (RP == 32) e = launch_forward<32>(P, ctas, st);
+    else e = launch_forward<64>(P, ctas, st);
     if (e != cudaSuccess) return e;
 
     const size_t gb = (size_t)BH * r * sizeof(float);
@@ -878,6 +993,6 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
     return cudaSuccess;
 }
 
-int fused_launches(int iters) { return 1 + (iters > 0 ? iters + 1 : 0) + 2; }
+int fused_launches(int iters) { (void)iters; return 2; }
 
 } // namespace lot
