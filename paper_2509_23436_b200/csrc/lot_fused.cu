@@ -16,21 +16,24 @@
 // out = softmax-rows x W' on tensor cores).
 //
 // Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-17 four epilogue
-// groups of 128 threads (tile k goes to group k % 4 and TMEM accumulator k % 4).  Producer and
-// MMA issuer never depend on G, so they run ahead across pass boundaries; only an epilogue
-// group waits, per segment, for the potential of that attempt.
+// groups of 128 threads (tile k goes to group k % 4 and TMEM accumulator k % 4), warp 18 the
+// reducer.  Producer and MMA issuer never depend on G, so they run ahead across pass
+// boundaries; only the epilogue warps wait, per segment, for the potential of that attempt.
 //
-// Cross-CTA protocol (all CTAs are co-resident: cooperative launch, one CTA per SM).  Every
-// group writes its column partial of a segment to its own slot and takes a ticket; the last
-// group to arrive merges all slots in slot order (deterministic), updates G and publishes
-// epoch = attempt + 1 with release semantics; waiters poll epoch with acquire loads.  Every
-// wait, on an mbarrier or on global memory, is bounded in time and raises LOT_DEV_TIMEOUT.
+// Cross-CTA protocol (all CTAs are co-resident: cooperative launch, one CTA per SM).  The
+// epilogue warps leave their column partials of a segment in shared memory and go on; the
+// reducer warp adds them in warp order, writes the CTA's partial to its slot and takes a
+// ticket; the reducer of the last CTA to arrive merges all slots in slot order (deterministic),
+// updates G and publishes epoch = attempt + 1 with release semantics; waiters poll epoch with
+// acquire loads.  Every wait, on an mbarrier or on global memory, is bounded in time and raises
+// LOT_DEV_TIMEOUT.
 #include "lot_common.cuh"
 #include "lot_internal.h"
 #include "lot_sm100.cuh"
 
 #include <cuda.h>
 #include <string.h>
+#include <type_traits>
 
 namespace lot {
 namespace fused {
@@ -40,7 +43,7 @@ using namespace sm100;
 constexpr int kPhaseSum = 0, kPhaseWred = 1, kPhaseOut = 2;
 constexpr int kGroups = 4;
 constexpr int kEpiThreads = kGroups * 128;
-constexpr int kThreads = 64 + kEpiThreads;
+constexpr int kThreads = 64 + kEpiThreads + 32;
 constexpr int kTileRows = 128;
 constexpr int kDK = 64;                          // head dimension of this path
 constexpr int kStageBytes = kTileRows * kDK * 2; // one token tile: 128 rows x 64 bf16, 128-byte swizzled
@@ -53,7 +56,7 @@ struct alignas(64) FusedParams {
     const float *beta;           // [H][r]
     const int32_t *key_len;      // [B] or nullptr
     float *G;                    // [2][BH][RP] pivot potentials, base-2 units (side 0 = queries, 1 = keys)
-    float *part;                 // [2][BH][maxslots*4][RP][2] column pairs per (CTA slot, group)
+    float *part;                 // [2][BH][maxslots][RP][2] column pairs per CTA slot
     unsigned *ticket;            // [2][BH]
     int *epoch;                  // [2][BH] attempts finished
     int *iter;                   // [2][BH] pivot updates done
@@ -134,8 +137,8 @@ struct Plan {
     static constexpr int offBar = offW + WBYTES;               // 64 mbarriers
     static constexpr int offMisc = offBar + 64 * 8;            // abort flag, TMEM base, flags
     static constexpr int offG = offMisc + 128;                 // float sG[4][64]
-    static constexpr int offRed = offG + kGroups * 64 * 4;     // float sRed[4][4][64][2]
-    static constexpr int total = offRed + kGroups * 4 * 64 * 2 * 4;
+    static constexpr int offPart = offG + kGroups * 64 * 4;    // float sPart[2][16][64][2]: per-warp column pairs
+    static constexpr int total = offPart + 2 * 16 * 64 * 2 * 4;
     static constexpr int dyn_bytes = total + 1024;             // slack for 1024-byte alignment
     static constexpr int tmem_cols = 512;
     static constexpr int colW = 256;                           // W accumulator (WRED): 64 columns
@@ -143,7 +146,8 @@ struct Plan {
 };
 
 enum BarId { bXFull = 0, bXEmpty = 8, bZFull = 16, bZEmpty = 18, bAccFull = 20, bAccEmpty = 24, bPFull = 28, bPEmpty = 30,
-             bOFull = 32, bOEmpty = 34, bWFull = 36, bWEmpty = 37, bWqFull = 38, bWqEmpty = 39, bCount = 40 };
+             bOFull = 32, bOEmpty = 34, bWFull = 36, bWEmpty = 37, bWqFull = 38, bWqEmpty = 39, bSegFull = 40, bSegEmpty = 42,
+             bCount = 44 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 {
@@ -232,11 +236,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     volatile int *sAbort = reinterpret_cast<volatile int *>(smem + PL::offMisc);
     uint32_t *sTmem = reinterpret_cast<uint32_t *>(smem + PL::offMisc + 4);
     volatile int *sLastW = reinterpret_cast<volatile int *>(smem + PL::offMisc + 8);
-    volatile int *sLast = reinterpret_cast<volatile int *>(smem + PL::offMisc + 16);   // [4]
-    volatile int *sFail = reinterpret_cast<volatile int *>(smem + PL::offMisc + 32);   // [4]
-    volatile int *sFlag = reinterpret_cast<volatile int *>(smem + PL::offMisc + 48);   // [4] per-group scratch flag
     float *sG = reinterpret_cast<float *>(smem + PL::offG);
-    float *sRed = reinterpret_cast<float *>(smem + PL::offRed);
+    float *sPart = reinterpret_cast<float *>(smem + PL::offPart);
     auto bar = [&](int id) { return smem_u32(bars + id); };
     // whole-warp wait with a warp-uniform verdict
     auto wwait = [&](uint32_t b, uint32_t parity) {
@@ -257,6 +258,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         for (int i = 0; i < kGroups; ++i) { mbar_init(bar(bAccFull + i), 1); mbar_init(bar(bAccEmpty + i), 4); }
         mbar_init(bar(bWFull), 1); mbar_init(bar(bWEmpty), 16);
         mbar_init(bar(bWqFull), 16); mbar_init(bar(bWqEmpty), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(bSegFull + i), 16); mbar_init(bar(bSegEmpty + i), 1); }
         *sAbort = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.tmQ); prefetch_tensormap(&P.tmK); prefetch_tensormap(&P.tmZ); prefetch_tensormap(&P.tmV);
@@ -442,7 +444,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         if (pend_k >= 0 && ok) issue_apply();
         if (w_open && ok && lane == 0) umma_commit(bar(bWFull));
         __syncwarp();
-    } else {
+    } else if (warp < 18) {
         // ======================= epilogue (16 warps, 4 groups) =======================
         const int ew = warp - 2, grp = ew >> 2, w4 = ew & 3, qd = warp & 3;
         const int etid = threadIdx.x - 64, gtid = w4 * 32 + lane;
@@ -450,201 +452,151 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         const int rit = qd * 32 + lane;                                   // row-per-thread layout: row inside the tile
         const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
         float *myG = sG + grp * 64;
-        float *myRed = sRed + grp * (4 * 64 * 2);
         Sched it(P);
         Seg g;
-        int k = 0, ka = 0, ko = 0, segw = 0, sego = 0;
+        int k = 0, ka = 0, ko = 0, segw = 0, sego = 0, segs = 0;
         bool ok = true;
 
         while (it.next(g)) {
             const int idx = g.side * BH + g.s;
-            // ---- wait until the potential this segment needs is published
-            if (gtid == 0) {
-                bool w = true;
-                if (g.phase == kPhaseSum) w = poll_ge(P.epoch + idx, g.attempt, sAbort, P.status);
-                else {
-                    w = poll_ge(P.iter + idx, P.T, sAbort, P.status);
-                    if (g.phase == kPhaseOut) {
-                        int kv = P.n;
-                        if (P.key_len != nullptr) kv = min(max(__ldg(P.key_len + g.b), 0), P.n);
-                        if (w && kv > 0) w = poll_ge(P.wdone + g.s, 1, sAbort, P.status);
-                    }
-                }
-                sFlag[grp] = (g.extra && w) ? __ldcg(P.robust + idx) : 1;
-            }
-            named_bar_sync(1 + grp, 128);
-            if (*sAbort) ok = false;
-            const int go = sFlag[grp];
-            const int rb = g.phase == kPhaseSum ? __ldcg(P.robust + idx) : 0;
-            named_bar_sync(1 + grp, 128);
-            if (g.extra && go == 0) continue;                           // this segment needed no repeat
-
             if (g.phase == kPhaseSum) {
                 // ================= SUM: quad layout, column sums in registers =================
-                float Gr[NC], acc[NC], kap[NC];
+                // every warp waits by itself for the potential of this attempt
+                int go = 0;
+                if (lane == 0) go = poll_ge(P.epoch + idx, g.attempt, sAbort, P.status) ? 1 + __ldcg(P.robust + idx) : 0;
+                go = __shfl_sync(0xffffffffu, go, 0);
+                if (go == 0) ok = false;
+                const int rb = go == 2;
+                if (g.extra && go == 1) continue;                       // this segment needed no repeat
+                float *dstp = sPart + (((segs & 1) * 16 + ew) * 64) * 2;
+                const uint32_t par_empty = ((segs >> 1) & 1) ^ 1;
+                const int par = segs & 1;
+                ++segs;
+
+                auto run = [&](auto rbtag) {
+                    constexpr bool RB = decltype(rbtag)::value;
+                    float Gr[NC], acc[NC], kap[RB ? NC : 1];
 #pragma unroll
-                for (int ci = 0; ci < NC; ++ci) {
-                    const int col = (ci >> 1) * 8 + 2 * cq + (ci & 1);
-                    Gr[ci] = col < P.r ? __ldcg(P.G + (size_t)idx * RP + col) : neg_inf();
-                    acc[ci] = 0.f; kap[ci] = neg_inf();
-                }
-                for (int t = g.t0; t < g.t1; ++t, ++k) {
-                    if ((k & 3) != grp) continue;
-                    const int j = k >> 2;
-                    if (ok) ok = wwait(bar(bAccFull + grp), j & 1);
-                    if (!ok) continue;
-                    tc_fence_after();
+                    for (int ci = 0; ci < NC; ++ci) {
+                        const int col = (ci >> 1) * 8 + 2 * cq + (ci & 1);
+                        Gr[ci] = col < P.r ? __ldcg(P.G + (size_t)idx * RP + col) : neg_inf();
+                        acc[ci] = 0.f;
+                        if (RB) kap[ci] = neg_inf();
+                    }
+                    for (int t = g.t0; t < g.t1; ++t, ++k) {
+                        if ((k & 3) != grp) continue;
+                        const int j = k >> 2;
+                        if (ok) ok = wwait(bar(bAccFull + grp), j & 1);
+                        if (!ok) continue;
+                        tc_fence_after();
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        float v[2 * NC];
-                        tmem_ld_quad<RP>(lane_addr + ((uint32_t)(half * 16) << 16) + grp * RP, v);
-                        tmem_wait_ld();
-                        if (half == 1) {
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(bar(bAccEmpty + grp));
-                        }
-                        const int rowA = t * kTileRows + qd * 32 + half * 16 + rq, rowB = rowA + 8;
-                        float mA = neg_inf(), mB = neg_inf();
-#pragma unroll
-                        for (int rep = 0; rep < NC / 2; ++rep) {
-                            v[rep * 4 + 0] += Gr[rep * 2]; v[rep * 4 + 1] += Gr[rep * 2 + 1];
-                            v[rep * 4 + 2] += Gr[rep * 2]; v[rep * 4 + 3] += Gr[rep * 2 + 1];
-                            mA = max3(mA, v[rep * 4 + 0], v[rep * 4 + 1]);
-                            mB = max3(mB, v[rep * 4 + 2], v[rep * 4 + 3]);
-                        }
-                        mA = fmaxf(mA, __shfl_xor_sync(0xffffffffu, mA, 1));
-                        mB = fmaxf(mB, __shfl_xor_sync(0xffffffffu, mB, 1));
-                        mA = fmaxf(mA, __shfl_xor_sync(0xffffffffu, mA, 2));
-                        mB = fmaxf(mB, __shfl_xor_sync(0xffffffffu, mB, 2));
-                        float sA0 = 0.f, sA1 = 0.f, sB0 = 0.f, sB1 = 0.f;
-                        if (!rb) {
+                        for (int half = 0; half < 2; ++half) {
+                            float v[2 * NC];
+                            tmem_ld_quad<RP>(lane_addr + ((uint32_t)(half * 16) << 16) + grp * RP, v);
+                            tmem_wait_ld();
+                            if (half == 1) {
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(bar(bAccEmpty + grp));
+                            }
+                            const int rowA = t * kTileRows + qd * 32 + half * 16 + rq, rowB = rowA + 8;
+                            float mA = neg_inf(), mB = neg_inf();
 #pragma unroll
                             for (int rep = 0; rep < NC / 2; ++rep) {
-                                v[rep * 4 + 0] = ex2(v[rep * 4 + 0] - mA); sA0 += v[rep * 4 + 0];
-                                v[rep * 4 + 1] = ex2(v[rep * 4 + 1] - mA); sA1 += v[rep * 4 + 1];
-                                v[rep * 4 + 2] = ex2(v[rep * 4 + 2] - mB); sB0 += v[rep * 4 + 2];
-                                v[rep * 4 + 3] = ex2(v[rep * 4 + 3] - mB); sB1 += v[rep * 4 + 3];
+                                v[rep * 4 + 0] += Gr[rep * 2]; v[rep * 4 + 1] += Gr[rep * 2 + 1];
+                                v[rep * 4 + 2] += Gr[rep * 2]; v[rep * 4 + 3] += Gr[rep * 2 + 1];
+                                mA = max3(mA, v[rep * 4 + 0], v[rep * 4 + 1]);
+                                mB = max3(mB, v[rep * 4 + 2], v[rep * 4 + 3]);
                             }
-                        } else {
+                            mA = fmaxf(mA, __shfl_xor_sync(0xffffffffu, mA, 1));
+                            mB = fmaxf(mB, __shfl_xor_sync(0xffffffffu, mB, 1));
+                            mA = fmaxf(mA, __shfl_xor_sync(0xffffffffu, mA, 2));
+                            mB = fmaxf(mB, __shfl_xor_sync(0xffffffffu, mB, 2));
+                            float sA0 = 0.f, sA1 = 0.f, sB0 = 0.f, sB1 = 0.f;
+                            if (!RB) {
 #pragma unroll
-                            for (int rep = 0; rep < NC / 2; ++rep) {
-                                sA0 += ex2(v[rep * 4 + 0] - mA); sA1 += ex2(v[rep * 4 + 1] - mA);
-                                sB0 += ex2(v[rep * 4 + 2] - mB); sB1 += ex2(v[rep * 4 + 3] - mB);
+                                for (int rep = 0; rep < NC / 2; ++rep) {
+                                    v[rep * 4 + 0] = ex2(v[rep * 4 + 0] - mA); sA0 += v[rep * 4 + 0];
+                                    v[rep * 4 + 1] = ex2(v[rep * 4 + 1] - mA); sA1 += v[rep * 4 + 1];
+                                    v[rep * 4 + 2] = ex2(v[rep * 4 + 2] - mB); sB0 += v[rep * 4 + 2];
+                                    v[rep * 4 + 3] = ex2(v[rep * 4 + 3] - mB); sB1 += v[rep * 4 + 3];
+                                }
+                            } else {
+#pragma unroll
+                                for (int rep = 0; rep < NC / 2; ++rep) {
+                                    sA0 += ex2(v[rep * 4 + 0] - mA); sA1 += ex2(v[rep * 4 + 1] - mA);
+                                    sB0 += ex2(v[rep * 4 + 2] - mB); sB1 += ex2(v[rep * 4 + 3] - mB);
+                                }
                             }
-                        }
-                        float sA = sA0 + sA1, sB = sB0 + sB1;
-                        sA += __shfl_xor_sync(0xffffffffu, sA, 1);
-                        sB += __shfl_xor_sync(0xffffffffu, sB, 1);
-                        sA += __shfl_xor_sync(0xffffffffu, sA, 2);
-                        sB += __shfl_xor_sync(0xffffffffu, sB, 2);
-                        if (!rb) {
-                            const float wA = rowA < g.nvalid ? __fdividef(1.f, sA) : 0.f;
-                            const float wB = rowB < g.nvalid ? __fdividef(1.f, sB) : 0.f;
+                            float sA = sA0 + sA1, sB = sB0 + sB1;
+                            sA += __shfl_xor_sync(0xffffffffu, sA, 1);
+                            sB += __shfl_xor_sync(0xffffffffu, sB, 1);
+                            sA += __shfl_xor_sync(0xffffffffu, sA, 2);
+                            sB += __shfl_xor_sync(0xffffffffu, sB, 2);
+                            if (!RB) {
+                                const float wA = rowA < g.nvalid ? __fdividef(1.f, sA) : 0.f;
+                                const float wB = rowB < g.nvalid ? __fdividef(1.f, sB) : 0.f;
 #pragma unroll
-                            for (int ci = 0; ci < NC; ++ci) {
-                                acc[ci] = fmaf(v[(ci >> 1) * 4 + (ci & 1)], wA, acc[ci]);
-                                acc[ci] = fmaf(v[(ci >> 1) * 4 + 2 + (ci & 1)], wB, acc[ci]);
-                            }
-                        } else {
-                            // exact log2 of every normalised entry, added to (kappa, S) pairs
-                            const float MA = mA + lg2(sA), MB = mB + lg2(sB);
+                                for (int ci = 0; ci < NC; ++ci) {
+                                    acc[ci] = fmaf(v[(ci >> 1) * 4 + (ci & 1)], wA, acc[ci]);
+                                    acc[ci] = fmaf(v[(ci >> 1) * 4 + 2 + (ci & 1)], wB, acc[ci]);
+                                }
+                            } else {
+                                // exact log2 of every normalised entry, added to (kappa, S) pairs
+                                const float MA = mA + lg2(sA), MB = mB + lg2(sB);
 #pragma unroll
-                            for (int ci = 0; ci < NC; ++ci) {
-                                const int col = (ci >> 1) * 8 + 2 * cq + (ci & 1);
-                                if (col < P.r) {
-                                    if (rowA < g.nvalid) pair_add(kap[ci], acc[ci], v[(ci >> 1) * 4 + (ci & 1)] - MA);
-                                    if (rowB < g.nvalid) pair_add(kap[ci], acc[ci], v[(ci >> 1) * 4 + 2 + (ci & 1)] - MB);
+                                for (int ci = 0; ci < NC; ++ci) {
+                                    const int col = (ci >> 1) * 8 + 2 * cq + (ci & 1);
+                                    if (col < P.r) {
+                                        if (rowA < g.nvalid) pair_add(kap[RB ? ci : 0], acc[ci], v[(ci >> 1) * 4 + (ci & 1)] - MA);
+                                        if (rowB < g.nvalid) pair_add(kap[RB ? ci : 0], acc[ci], v[(ci >> 1) * 4 + 2 + (ci & 1)] - MB);
+                                    }
                                 }
                             }
                         }
                     }
-                }
-                // ---- group partial: rows of the warp (lanes with equal cq), then the 4 warps
+                    // ---- warp partial: the 8 rows-lanes of every column quarter, left in shared memory
 #pragma unroll
-                for (int off = 4; off <= 16; off <<= 1) {
+                    for (int off = 4; off <= 16; off <<= 1) {
 #pragma unroll
-                    for (int ci = 0; ci < NC; ++ci) {
-                        if (rb) {
-                            const float ok2 = __shfl_xor_sync(0xffffffffu, kap[ci], off);
-                            const float os2 = __shfl_xor_sync(0xffffffffu, acc[ci], off);
-                            pair_merge(kap[ci], acc[ci], ok2, os2);
-                        } else {
-                            acc[ci] += __shfl_xor_sync(0xffffffffu, acc[ci], off);
+                        for (int ci = 0; ci < NC; ++ci) {
+                            if (RB) {
+                                const float ok2 = __shfl_xor_sync(0xffffffffu, kap[RB ? ci : 0], off);
+                                const float os2 = __shfl_xor_sync(0xffffffffu, acc[ci], off);
+                                pair_merge(kap[RB ? ci : 0], acc[ci], ok2, os2);
+                            } else {
+                                acc[ci] += __shfl_xor_sync(0xffffffffu, acc[ci], off);
+                            }
                         }
                     }
-                }
-                if (rq == 0) {
+                    if (ok) ok = wwait(bar(bSegEmpty + par), par_empty);
+                    if (rq == 0) {
 #pragma unroll
-                    for (int ci = 0; ci < NC; ++ci) {
-                        const int col = (ci >> 1) * 8 + 2 * cq + (ci & 1);
-                        myRed[(w4 * 64 + col) * 2] = rb ? kap[ci] : 0.f;
-                        myRed[(w4 * 64 + col) * 2 + 1] = acc[ci];
-                    }
-                }
-                named_bar_sync(1 + grp, 128);
-                if (gtid < RP) {
-                    float kk = myRed[gtid * 2], ss = myRed[gtid * 2 + 1];
-#pragma unroll
-                    for (int w = 1; w < 4; ++w) {
-                        if (rb) pair_merge(kk, ss, myRed[(w * 64 + gtid) * 2], myRed[(w * 64 + gtid) * 2 + 1]);
-                        else ss += myRed[(w * 64 + gtid) * 2 + 1];
-                    }
-                    float *dst = P.part + ((((size_t)idx * P.maxslots + g.slot) * 4 + grp) * RP + gtid) * 2;
-                    __stcg(reinterpret_cast<float2 *>(dst), make_float2(kk, ss));
-                    __threadfence();
-                }
-                named_bar_sync(1 + grp, 128);
-                if (gtid == 0) {
-                    __threadfence();
-                    const unsigned tk = atomicAdd(P.ticket + idx, 1u);
-                    sLast[grp] = (tk == (unsigned)(g.nslots * 4) - 1u);
-                    sFail[grp] = 0;
-                }
-                named_bar_sync(1 + grp, 128);
-                if (sLast[grp]) {
-                    // ---- last group of the (slice, side): merge every slot in slot order, update G
-                    __threadfence();
-                    const int nparts = g.nslots * 4;
-                    const int col = gtid & 63, hsel = gtid >> 6;
-                    float kk = rb ? neg_inf() : 0.f, ss = 0.f;
-                    if (col < RP) {
-                        const float *src = P.part + ((size_t)idx * P.maxslots * 4) * RP * 2 + col * 2;
-                        for (int p = hsel; p < nparts; p += 2) {
-                            const float2 pr = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)p * RP * 2));
-                            if (rb) pair_merge(kk, ss, pr.x, pr.y);
-                            else ss += pr.y;
+                        for (int ci = 0; ci < NC; ci += 2) {
+                            const int col = (ci >> 1) * 8 + 2 * cq;
+                            *reinterpret_cast<float4 *>(dstp + col * 2) =
+                                make_float4(RB ? kap[RB ? ci : 0] : 0.f, acc[ci], RB ? kap[RB ? ci + 1 : 0] : 0.f, acc[ci + 1]);
                         }
                     }
-                    if (hsel == 1) { myRed[col * 2] = kk; myRed[col * 2 + 1] = ss; }
-                    named_bar_sync(1 + grp, 128);
-                    if (hsel == 0 && col < P.r) {
-                        if (rb) pair_merge(kk, ss, myRed[col * 2], myRed[col * 2 + 1]);
-                        else ss += myRed[col * 2 + 1];
-                        if (!rb && !(ss >= kPlainFloor && ss <= 3.0e38f)) sFail[grp] = 1;
-                    }
-                    named_bar_sync(1 + grp, 128);
-                    const int fail = sFail[grp];
-                    const int itn = __ldcg(P.iter + idx);
-                    if (!fail && hsel == 0 && col < P.r) {
-                        float *gp = P.G + (size_t)idx * RP + col;
-                        const float gn = __ldcg(gp) + lg2(__ldg(P.beta + g.h * P.r + col) * (float)g.nvalid) - (kk + lg2(ss));
-                        if (!isfinite(gn)) atomicOr(P.status, 1 /* LOT_DEV_NONFINITE */);
-                        __stcg(gp, gn);
-                        if (itn + 1 == P.T) P.g_nat[(size_t)idx * P.r + col] = gn * P.eps_ln2;
-                        __threadfence();
-                    }
-                    named_bar_sync(1 + grp, 128);
-                    if (gtid == 0) {
-                        __stcg(P.ticket + idx, 0u);
-                        if (fail) __stcg(P.robust + idx, 1);
-                        __threadfence();
-                        if (!fail) st_release(P.iter + idx, itn + 1);
-                        st_release(P.epoch + idx, g.attempt + 1);
-                    }
-                }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(bSegFull + par));
+                };
+                if (rb) run(std::true_type{});
+                else run(std::false_type{});
                 continue;
             }
+
+            // ---- WRED / OUT: wait until the final potential (and W') of this slice is published
+            if (gtid == 0) {
+                bool w = poll_ge(P.iter + idx, P.T, sAbort, P.status);
+                if (g.phase == kPhaseOut) {
+                    int kv = P.n;
+                    if (P.key_len != nullptr) kv = min(max(__ldg(P.key_len + g.b), 0), P.n);
+                    if (w && kv > 0) w = poll_ge(P.wdone + g.s, 1, sAbort, P.status);
+                }
+            }
+            named_bar_sync(1 + grp, 128);
+            if (*sAbort) ok = false;
 
             // ================= WRED / OUT: one thread per token row =================
             if (gtid < RP) myG[gtid] = gtid < P.r ? __ldcg(P.G + (size_t)idx * RP + gtid) : neg_inf();
@@ -773,18 +725,37 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 if (*sLastW) {
                     __threadfence();
                     const float mass = g.nvalid > 0 ? 1.f / (float)g.nvalid : 0.f;
-                    for (int e = etid; e < 64 * DK; e += kEpiThreads) {
-                        const int tt = e / DK, c = e % DK;
-                        float sum = 0.f;
-                        for (int sl = 0; sl < g.nslots; ++sl) {
-                            const float *src = P.wpart + (((size_t)g.s * P.maxslots + sl) * 128) * DK + c;
-                            sum += __ldcg(src + (size_t)tt * DK) + __ldcg(src + (size_t)(64 + tt) * DK);
+                    // 64 pivots x 64 channels, four channels per thread; slots in order, four slots of loads in flight
+                    for (int e = etid; e < 64 * DK / 4; e += kEpiThreads) {
+                        const int tt = e / (DK / 4), c = (e % (DK / 4)) * 4;
+                        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+                        const float *src0 = P.wpart + ((size_t)g.s * P.maxslots * 128) * DK + c;
+                        for (int sl0 = 0; sl0 < g.nslots; sl0 += 4) {
+                            float4 a[4], b[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                a[u] = b[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (sl0 + u < g.nslots) {
+                                    const float *src = src0 + ((size_t)(sl0 + u) * 128) * DK;
+                                    a[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)tt * DK));
+                                    b[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(64 + tt) * DK));
+                                }
+                            }
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                sum.x += a[u].x + b[u].x; sum.y += a[u].y + b[u].y;
+                                sum.z += a[u].z + b[u].z; sum.w += a[u].w + b[u].w;
+                            }
                         }
-                        const float wv = tt < P.r ? sum * mass / __ldg(P.beta + g.h * P.r + tt) : 0.f;
-                        const __nv_bfloat16 hi = __float2bfloat16_rn(wv);
-                        const __nv_bfloat16 lo = __float2bfloat16_rn(wv - __bfloat162float(hi));
-                        P.Wb[(((size_t)g.s * 2 + 0) * DK + c) * 64 + tt] = hi;
-                        P.Wb[(((size_t)g.s * 2 + 1) * DK + c) * 64 + tt] = lo;
+                        const float sc = tt < P.r ? mass / __ldg(P.beta + g.h * P.r + tt) : 0.f;
+                        const float wv[4] = {sum.x * sc, sum.y * sc, sum.z * sc, sum.w * sc};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const __nv_bfloat16 hi = __float2bfloat16_rn(wv[u]);
+                            const __nv_bfloat16 lo = __float2bfloat16_rn(wv[u] - __bfloat162float(hi));
+                            P.Wb[(((size_t)g.s * 2 + 0) * DK + c + u) * 64 + tt] = hi;
+                            P.Wb[(((size_t)g.s * 2 + 1) * DK + c + u) * 64 + tt] = lo;
+                        }
                     }
                     __threadfence();
                     named_bar_sync(5, kEpiThreads);
@@ -794,6 +765,106 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         st_release(P.wdone + g.s, 1);
                     }
                 }
+            }
+        }
+    } else {
+        // ======================= reducer (one warp): CTA partials, tickets, pivot updates =======================
+        Sched it(P);
+        Seg g;
+        int segs = 0;
+        bool ok = true;
+        const int c0 = 2 * lane;                          // this lane's two columns (lanes with c0 >= RP idle)
+        const bool mine = c0 < RP;
+        while (it.next(g)) {
+            if (g.phase != kPhaseSum) break;              // SUM segments come first in the schedule
+            const int idx = g.side * BH + g.s;
+            int rb = __ldcg(P.robust + idx);              // stable once the segment's attempt has been reached
+            if (g.extra) {
+                int go = 0;
+                if (lane == 0) go = poll_ge(P.epoch + idx, P.T, sAbort, P.status) ? 1 + __ldcg(P.robust + idx) : 0;
+                go = __shfl_sync(0xffffffffu, go, 0);
+                if (go == 0) ok = false;
+                if (go == 1) continue;
+                rb = 1;
+            }
+            const int par = segs & 1;
+            if (ok) ok = wwait(bar(bSegFull + par), (segs >> 1) & 1);
+            ++segs;
+            if (!ok) continue;
+            // the epilogue warps read robust after their own epoch wait; re-read it now that they have arrived
+            rb = __ldcg(P.robust + idx);
+            float k0 = rb ? neg_inf() : 0.f, s0 = 0.f, k1 = k0, s1 = 0.f;
+            if (mine) {
+                const float *src = sPart + ((par * 16) * 64 + c0) * 2;
+#pragma unroll
+                for (int w = 0; w < 16; ++w) {
+                    const float4 pr = *reinterpret_cast<const float4 *>(src + w * 128);
+                    if (rb) { pair_merge(k0, s0, pr.x, pr.y); pair_merge(k1, s1, pr.z, pr.w); }
+                    else { s0 += pr.y; s1 += pr.w; }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(bSegEmpty + par));
+            if (mine)
+                __stcg(reinterpret_cast<float4 *>(P.part + (((size_t)idx * P.maxslots + g.slot) * RP + c0) * 2),
+                       make_float4(k0, s0, k1, s1));
+            __threadfence();
+            __syncwarp();
+            int last = 0;
+            if (lane == 0) {
+                __threadfence();
+                last = atomicAdd(P.ticket + idx, 1u) == (unsigned)g.nslots - 1u;
+            }
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (!last) continue;
+            // ---- last CTA of the (slice, side): merge every slot in slot order, update G
+            __threadfence();
+            k0 = k1 = rb ? neg_inf() : 0.f; s0 = s1 = 0.f;
+            if (mine) {
+                const float *src = P.part + ((size_t)idx * P.maxslots * RP + c0) * 2;
+                for (int p0 = 0; p0 < g.nslots; p0 += 8) {
+                    float4 pr[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        pr[u] = make_float4(neg_inf(), 0.f, neg_inf(), 0.f);
+                        if (p0 + u < g.nslots) pr[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(p0 + u) * RP * 2));
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (rb) { pair_merge(k0, s0, pr[u].x, pr[u].y); pair_merge(k1, s1, pr[u].z, pr[u].w); }
+                        else { s0 += pr[u].y; s1 += pr[u].w; }
+                    }
+                }
+            }
+            bool bad = false;
+            if (!rb && mine) {
+                if (c0 < P.r && !(s0 >= kPlainFloor && s0 <= 3.0e38f)) bad = true;
+                if (c0 + 1 < P.r && !(s1 >= kPlainFloor && s1 <= 3.0e38f)) bad = true;
+            }
+            const int fail = __any_sync(0xffffffffu, bad);
+            const int itn = __ldcg(P.iter + idx);
+            if (!fail && mine) {
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int col = c0 + u;
+                    if (col < P.r) {
+                        float *gp = P.G + (size_t)idx * RP + col;
+                        const float kk = u ? k1 : k0, ss = u ? s1 : s0;
+                        const float gn = __ldcg(gp) + lg2(__ldg(P.beta + g.h * P.r + col) * (float)g.nvalid) - (kk + lg2(ss));
+                        if (!isfinite(gn)) atomicOr(P.status, 1 /* LOT_DEV_NONFINITE */);
+                        __stcg(gp, gn);
+                        if (itn + 1 == P.T) P.g_nat[(size_t)idx * P.r + col] = gn * P.eps_ln2;
+                    }
+                }
+                __threadfence();
+            }
+            __syncwarp();
+            if (lane == 0) {
+                __stcg(P.ticket + idx, 0u);
+                if (fail) __stcg(P.robust + idx, 1);
+                __threadfence();
+                if (!fail) st_release(P.iter + idx, itn + 1);
+                st_release(P.epoch + idx, g.attempt + 1);
             }
         }
     }
@@ -918,7 +989,7 @@ FusedLayout fused_layout(int B, int H, int n, int d, int r)
     L.Wb = o; o += up256((size_t)BH * 2 * d * 64 * 2);
     L.head_end = o;
     L.zprep = o; o += up256((size_t)H * 2 * RP * d * 2);
-    L.part = o; o += up256((size_t)2 * BH * ms * 4 * RP * 2 * 4);
+    L.part = o; o += up256((size_t)2 * BH * ms * RP * 2 * 4);
     L.wpart = o; o += up256((size_t)BH * ms * 128 * d * 4);
     L.total = o;
     return L;
