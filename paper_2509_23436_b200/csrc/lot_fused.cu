@@ -17,16 +17,19 @@
 //
 // Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-17 four epilogue
 // groups of 128 threads (tile k goes to group k % 4 and TMEM accumulator k % 4), warp 18 the
-// reducer.  Producer and MMA issuer never depend on G, so they run ahead across pass
-// boundaries; only the epilogue warps wait, per segment, for the potential of that attempt.
+// publisher, warp 19 the gatherer.  Producer and MMA issuer never depend on G, so they run
+// ahead across pass boundaries; only the epilogue warps wait, per segment, for the potential of
+// that attempt.
 //
 // Cross-CTA protocol (all CTAs are co-resident: cooperative launch, one CTA per SM).  The
 // epilogue warps leave their column partials of a segment in shared memory and go on; the
-// reducer warp adds them in warp order, writes the CTA's partial to its slot and takes a
-// ticket; the reducer of the last CTA to arrive merges all slots in slot order (deterministic),
-// updates G and publishes epoch = attempt + 1 with release semantics; waiters poll epoch with
-// acquire loads.  Every wait, on an mbarrier or on global memory, is bounded in time and raises
-// LOT_DEV_TIMEOUT.
+// publisher warp adds them in warp order and writes the CTA's partial to its slot as 64-bit
+// words that carry the attempt number beside the value, so a word is valid by itself and no
+// fence or ticket is needed.  The gatherer warp of EVERY CTA that shares the (slice, side) polls
+// all slots until their tags match, merges them in slot order (deterministic and identical in
+// all CTAs, including the verdict that plain sums underflowed), updates its copy of G and hands
+// it to its epilogue warps through shared memory.  Every wait, on an mbarrier, on shared or on
+// global memory, is bounded in time and raises LOT_DEV_TIMEOUT.
 #include "lot_common.cuh"
 #include "lot_internal.h"
 #include "lot_sm100.cuh"
@@ -43,7 +46,8 @@ using namespace sm100;
 constexpr int kPhaseSum = 0, kPhaseWred = 1, kPhaseOut = 2;
 constexpr int kGroups = 4;
 constexpr int kEpiThreads = kGroups * 128;
-constexpr int kThreads = 64 + kEpiThreads + 32;
+constexpr int kThreads = 64 + kEpiThreads + 64;
+constexpr int kMaxLoc = 16;                      // (slice, side) states of a CTA cached in shared memory
 constexpr int kTileRows = 128;
 constexpr int kDK = 64;                          // head dimension of this path
 constexpr int kStageBytes = kTileRows * kDK * 2; // one token tile: 128 rows x 64 bf16, 128-byte swizzled
@@ -56,9 +60,8 @@ struct alignas(64) FusedParams {
     const float *beta;           // [H][r]
     const int32_t *key_len;      // [B] or nullptr
     float *G;                    // [2][BH][RP] pivot potentials, base-2 units (side 0 = queries, 1 = keys)
-    float *part;                 // [2][BH][maxslots][RP][2] column pairs per CTA slot
-    unsigned *ticket;            // [2][BH]
-    int *epoch;                  // [2][BH] attempts finished
+    unsigned long long *part;    // [2 attempt parities][2][BH][maxslots][RP][2] tagged words per CTA slot: (kappa, tag), (S, tag)
+    int *epoch;                  // [2][BH] attempts finished (used for segments beyond the shared-memory cache)
     int *iter;                   // [2][BH] pivot updates done
     int *robust;                 // [2][BH] 1 = column sums carried as (kappa, S) pairs (sticky)
     float *wpart;                // [BH][maxslots][128][64] per-slot W accumulators (rows 0-63 hi, 64-127 lo)
@@ -97,6 +100,8 @@ struct Sched {
         s = s_lo;
         side_idx = 0;
     }
+    // index of the (slice, side) among this CTA's segments of one pass
+    __device__ int local(const Seg &g) const { return (g.s - s_lo) * 2 + (g.side ? 0 : 1); }
     __device__ bool next(Seg &g)
     {
         for (;;) {
@@ -137,8 +142,12 @@ struct Plan {
     static constexpr int offBar = offW + WBYTES;               // 64 mbarriers
     static constexpr int offMisc = offBar + 64 * 8;            // abort flag, TMEM base, flags
     static constexpr int offG = offMisc + 128;                 // float sG[4][64]
-    static constexpr int offPart = offG + kGroups * 64 * 4;    // float sPart[2][16][64][2]: per-warp column pairs
-    static constexpr int total = offPart + 2 * 16 * 64 * 2 * 4;
+    static constexpr int offGc = offG + kGroups * 64 * 4;      // float sGc[kMaxLoc][64]: this CTA's copy of the potentials
+    static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust [kMaxLoc]
+    static constexpr int total = offState + 3 * kMaxLoc * 4;
+    // float sPart[2][16][64][2], the per-warp column pairs of the SUM passes, lives in the first plan buffer
+    // (free until the WRED pass; the epilogue waits for the publisher's last read before it writes a plan tile)
+    static constexpr int offPart = offP;
     static constexpr int dyn_bytes = total + 1024;             // slack for 1024-byte alignment
     static constexpr int tmem_cols = 512;
     static constexpr int colW = 256;                           // W accumulator (WRED): 64 columns
@@ -190,6 +199,35 @@ __device__ __forceinline__ bool poll_ge(const int *p, int want, volatile int *ab
     return false;
 }
 
+// The same on a shared-memory word written by another warp of this CTA.
+__device__ __forceinline__ bool spin_ge(volatile int *p, int want, volatile int *abort_flag, int *status)
+{
+    if (*abort_flag) return false;
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (*p >= want) return true;
+        if ((it & 255u) == 255u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
+        }
+    }
+    *abort_flag = 1;
+    atomicOr(status, 4 /* LOT_DEV_TIMEOUT */);
+    return false;
+}
+__device__ __forceinline__ void st_tagged(unsigned long long *p, float a, float b, unsigned tag)
+{
+    const unsigned long long w0 = ((unsigned long long)tag << 32) | __float_as_uint(a);
+    const unsigned long long w1 = ((unsigned long long)tag << 32) | __float_as_uint(b);
+    asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};" ::"l"(p), "l"(w0), "l"(w1) : "memory");
+}
+__device__ __forceinline__ void ld_tagged(const unsigned long long *p, unsigned long long &w0, unsigned long long &w1)
+{
+    asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(p) : "memory");
+}
+
 // Quad-layout TMEM load (16 lanes x RP columns): thread L of the warp gets, in v[rep*4 + k],
 // lane L/4 + 8*(k/2) and column rep*8 + 2*(L%4) + (k%2) of the 16-lane block at taddr.
 template <int RP>
@@ -238,6 +276,16 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     volatile int *sLastW = reinterpret_cast<volatile int *>(smem + PL::offMisc + 8);
     float *sG = reinterpret_cast<float *>(smem + PL::offG);
     float *sPart = reinterpret_cast<float *>(smem + PL::offPart);
+    float *sGc = reinterpret_cast<float *>(smem + PL::offGc);
+    volatile int *sDone = reinterpret_cast<volatile int *>(smem + PL::offState);
+    volatile int *sIter = sDone + kMaxLoc;
+    volatile int *sRobust = sIter + kMaxLoc;
+    volatile int *sPubDone = reinterpret_cast<volatile int *>(smem + PL::offMisc + 12);
+    // Wait until `need` attempts of local segment li (global index idx) are complete: 0 = gave up, else 1 + robust flag
+    auto seg_state = [&](int li, int idx, int need) -> int {
+        if (li < kMaxLoc) return spin_ge(sDone + li, need, sAbort, P.status) ? 1 + sRobust[li] : 0;
+        return poll_ge(P.epoch + idx, need, sAbort, P.status) ? 1 + __ldcg(P.robust + idx) : 0;
+    };
     auto bar = [&](int id) { return smem_u32(bars + id); };
     // whole-warp wait with a warp-uniform verdict
     auto wwait = [&](uint32_t b, uint32_t parity) {
@@ -260,10 +308,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         mbar_init(bar(bWqFull), 16); mbar_init(bar(bWqEmpty), 1);
         for (int i = 0; i < 2; ++i) { mbar_init(bar(bSegFull + i), 16); mbar_init(bar(bSegEmpty + i), 1); }
         *sAbort = 0;
+        *sPubDone = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.tmQ); prefetch_tensormap(&P.tmK); prefetch_tensormap(&P.tmZ); prefetch_tensormap(&P.tmV);
     }
     if (warp == 1) { tmem_alloc(smem_u32(sTmem), PL::tmem_cols); tmem_relinquish(); }
+    for (int i = threadIdx.x; i < kMaxLoc * 64; i += kThreads) sGc[i] = 0.f;
+    if (threadIdx.x < 3 * kMaxLoc) sDone[threadIdx.x] = 0;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -283,9 +334,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             while (ok && it.next(g)) {
                 const int idx = g.side * BH + g.s;
                 if (g.extra) {
-                    ok = poll_ge(P.epoch + idx, P.T, sAbort, P.status);
-                    if (!ok) break;
-                    if (__ldcg(P.robust + idx) == 0) continue;
+                    const int go = seg_state(it.local(g), idx, P.T);
+                    if (go == 0) { ok = false; break; }
+                    if (go == 1) continue;
                 }
                 const int zs = g.h & 1;
                 if (ztag[zs] != g.h) {
@@ -331,44 +382,50 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         __syncwarp();
     } else if (warp == 1) {
         // ======================= MMA issuer =======================
+        // The whole warp runs the loop with warp-uniform values (so that descriptors and addresses can stay in
+        // uniform registers); one elected lane issues the tcgen05 instructions.
         Sched it(P);
         Seg g;
         int k = 0, kx = 0, ztag[2] = {-1, -1}, zuse[2] = {0, 0}, segw = 0, sego = 0;
         int ka = 0, ko = 0;                   // tiles of the apply passes / of the OUT pass so far
         bool ok = true, w_open = false;
         int pend_k = -1, pend_o = 0, pend_first = 0, pend_vs = 0, pend_phase = 0;   // apply MMA still to be issued
+        const uint32_t tm = __shfl_sync(0xffffffffu, tmem_base, 0);
+        // Descriptors differ only in the 16-byte-granular start address (low word).
+        const uint64_t dK = make_smem_desc(sbase, 16, 1024);               // K-major operand, 128-byte rows
+        const uint64_t dMN = make_smem_desc(sbase, kStageBytes, 1024);     // MN-major operand, panels kStageBytes apart
+        const uint32_t dK_hi = (uint32_t)(dK >> 32), dK_lo = (uint32_t)dK;
+        const uint32_t dMN_hi = (uint32_t)(dMN >> 32), dMN_lo = (uint32_t)dMN;
+        auto desc = [](uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
 
         auto issue_apply = [&]() {
             const int pb = pend_k & 1, pj = pend_k >> 1, ob = pend_o & 1, oj = pend_o >> 1;
             if (ok) ok = wwait(bar(bPFull + pb), pj & 1);
-            const uint32_t pa = sbase + PL::offP + pb * PL::PBYTES;
+            const uint32_t pa = (PL::offP + pb * PL::PBYTES) >> 4;
             if (pend_phase == kPhaseWred) {
                 const int vs = pend_vs % kStages, vph = (pend_vs / kStages) & 1;
                 if (ok) ok = wwait(bar(bXFull + vs), vph);
                 tc_fence_after();
-                if (ok && lane == 0) {
-                    const uint32_t va = sbase + PL::offX + vs * kStageBytes;
+                const uint32_t va = (PL::offX + vs * kStageBytes) >> 4;
+                if (ok && elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        uint64_t ad = make_smem_desc(pa + ks * 2048, kStageBytes, 1024);
-                        uint64_t bd = make_smem_desc(va + ks * 2048, kStageBytes, 1024);
-                        umma_bf16(tmem_base + PL::colW, ad, bd, idesc_w, (pend_first && ks == 0) ? 0u : 1u);
-                    }
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_bf16(tm + PL::colW, desc(dMN_hi, dMN_lo + pa + ks * 128),
+                                  desc(dMN_hi, dMN_lo + va + ks * 128), idesc_w, (pend_first && ks == 0) ? 0u : 1u);
                     umma_commit(bar(bPEmpty + pb));
                     umma_commit(bar(bXEmpty + vs));
                 }
             } else {
                 if (ok) ok = wwait(bar(bOEmpty + ob), (oj & 1) ^ 1);
                 tc_fence_after();
-                if (ok && lane == 0) {
+                if (ok && elect_one()) {
 #pragma unroll
                     for (int part = 0; part < 2; ++part)
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {
-                            uint64_t ad = make_smem_desc(pa + ks * 32, 16, 1024);
-                            uint64_t bd = make_smem_desc(sbase + PL::offW + part * (DK * 128) + ks * 32, 16, 1024);
-                            umma_bf16(tmem_base + PL::colO + ob * DK, ad, bd, idesc_o, (part | ks) ? 1u : 0u);
-                        }
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_bf16(tm + PL::colO + ob * DK, desc(dK_hi, dK_lo + pa + ks * 2),
+                                      desc(dK_hi, dK_lo + ((PL::offW + part * (DK * 128)) >> 4) + ks * 2), idesc_o,
+                                      (part | ks) ? 1u : 0u);
                     umma_commit(bar(bPEmpty + pb));
                     umma_commit(bar(bOFull + ob));
                 }
@@ -381,14 +438,14 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             const int idx = g.side * BH + g.s;
             if (g.extra) {
                 int go = 0;
-                if (lane == 0) go = poll_ge(P.epoch + idx, P.T, sAbort, P.status) ? (__ldcg(P.robust + idx) ? 2 : 1) : 0;
+                if (lane == 0) go = seg_state(it.local(g), idx, P.T);
                 go = __shfl_sync(0xffffffffu, go, 0);
                 if (go == 0) { ok = false; break; }
                 if (go == 1) continue;
             }
             if (pend_k >= 0) issue_apply();
             if (w_open) {                                                    // W of the previous WRED segment complete
-                if (ok && lane == 0) umma_commit(bar(bWFull));
+                if (ok && elect_one()) umma_commit(bar(bWFull));
                 __syncwarp();
                 w_open = false;
             }
@@ -399,34 +456,33 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             }
             const int zs = g.h & 1;
             if (ztag[zs] != g.h) {
-                if (zuse[zs] > 0 && lane == 0) umma_commit(bar(bZEmpty + zs));
+                if (zuse[zs] > 0 && elect_one()) umma_commit(bar(bZEmpty + zs));
                 __syncwarp();
                 if (ok) ok = wwait(bar(bZFull + zs), zuse[zs] & 1);
                 ztag[zs] = g.h; ++zuse[zs];
             }
             if (g.phase == kPhaseOut) {
-                if (sego > 0 && lane == 0) umma_commit(bar(bWqEmpty));
+                if (sego > 0 && elect_one()) umma_commit(bar(bWqEmpty));
                 __syncwarp();
                 if (ok) ok = wwait(bar(bWqFull), sego & 1);
                 ++sego;
             }
+            const uint32_t za = dK_lo + ((PL::offZ + zs * PL::ZBYTES) >> 4);
             for (int t = g.t0; t < g.t1 && ok; ++t, ++k) {
                 const int grp = k & 3, j = k >> 2;
                 const int st = kx % kStages, ph = (kx / kStages) & 1;
                 ok = wwait(bar(bXFull + st), ph);
                 if (ok) ok = wwait(bar(bAccEmpty + grp), (j & 1) ^ 1);
                 tc_fence_after();
-                if (ok && lane == 0) {
-                    const uint32_t xa = sbase + PL::offX + st * kStageBytes;
-                    const uint32_t za = sbase + PL::offZ + zs * PL::ZBYTES;
+                const uint32_t xa = dK_lo + ((PL::offX + st * kStageBytes) >> 4);
+                const uint32_t dcol = tm + grp * RP;
+                if (ok && elect_one()) {
 #pragma unroll
                     for (int part = 0; part < 2; ++part)
 #pragma unroll
-                        for (int kk = 0; kk < DK / 16; ++kk) {
-                            uint64_t ad = make_smem_desc(xa + kk * 32, 16, 1024);
-                            uint64_t bd = make_smem_desc(za + part * (64 * 128) + kk * 32, 16, 1024);
-                            umma_bf16(tmem_base + grp * RP, ad, bd, idesc_cost, (part | kk) ? 1u : 0u);
-                        }
+                        for (int kk = 0; kk < DK / 16; ++kk)
+                            umma_bf16(dcol, desc(dK_hi, xa + kk * 2), desc(dK_hi, za + part * ((64 * 128) >> 4) + kk * 2),
+                                      idesc_cost, (part | kk) ? 1u : 0u);
                     umma_commit(bar(bXEmpty + st));
                     umma_commit(bar(bAccFull + grp));
                 }
@@ -442,7 +498,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             }
         }
         if (pend_k >= 0 && ok) issue_apply();
-        if (w_open && ok && lane == 0) umma_commit(bar(bWFull));
+        if (w_open && ok && elect_one()) umma_commit(bar(bWFull));
         __syncwarp();
     } else if (warp < 18) {
         // ======================= epilogue (16 warps, 4 groups) =======================
@@ -462,8 +518,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             if (g.phase == kPhaseSum) {
                 // ================= SUM: quad layout, column sums in registers =================
                 // every warp waits by itself for the potential of this attempt
+                const int li = it.local(g);
                 int go = 0;
-                if (lane == 0) go = poll_ge(P.epoch + idx, g.attempt, sAbort, P.status) ? 1 + __ldcg(P.robust + idx) : 0;
+                if (lane == 0) go = seg_state(li, idx, g.attempt);
                 go = __shfl_sync(0xffffffffu, go, 0);
                 if (go == 0) ok = false;
                 const int rb = go == 2;
@@ -479,7 +536,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
 #pragma unroll
                     for (int ci = 0; ci < NC; ++ci) {
                         const int col = (ci >> 1) * 8 + 2 * cq + (ci & 1);
-                        Gr[ci] = col < P.r ? __ldcg(P.G + (size_t)idx * RP + col) : neg_inf();
+                        Gr[ci] = col < P.r ? (li < kMaxLoc ? sGc[li * 64 + col] : __ldcg(P.G + (size_t)idx * RP + col)) : neg_inf();
                         acc[ci] = 0.f;
                         if (RB) kap[ci] = neg_inf();
                     }
@@ -586,9 +643,11 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 continue;
             }
 
-            // ---- WRED / OUT: wait until the final potential (and W') of this slice is published
+            // ---- WRED / OUT: wait until the final potential (and W') of this slice is known here
+            const int li = it.local(g);
             if (gtid == 0) {
-                bool w = poll_ge(P.iter + idx, P.T, sAbort, P.status);
+                bool w = spin_ge(sPubDone, 1, sAbort, P.status);          // plan buffers free of SUM partials
+                if (w) w = li < kMaxLoc ? spin_ge(sIter + li, P.T, sAbort, P.status) : poll_ge(P.iter + idx, P.T, sAbort, P.status);
                 if (g.phase == kPhaseOut) {
                     int kv = P.n;
                     if (P.key_len != nullptr) kv = min(max(__ldg(P.key_len + g.b), 0), P.n);
@@ -599,7 +658,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             if (*sAbort) ok = false;
 
             // ================= WRED / OUT: one thread per token row =================
-            if (gtid < RP) myG[gtid] = gtid < P.r ? __ldcg(P.G + (size_t)idx * RP + gtid) : neg_inf();
+            if (gtid < RP)
+                myG[gtid] = gtid < P.r ? (li < kMaxLoc ? sGc[li * 64 + gtid] : __ldcg(P.G + (size_t)idx * RP + gtid)) : neg_inf();
             if (g.phase == kPhaseOut) {
                 // stage W'^T (hi, lo) of this slice as the B operand: 128-byte rows, 16-byte chunks xor row%8
                 if (sego > 0 && ok) ok = wwait(bar(bWqEmpty), (sego - 1) & 1);
@@ -767,8 +827,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 }
             }
         }
-    } else {
-        // ======================= reducer (one warp): CTA partials, tickets, pivot updates =======================
+    } else if (warp == 18) {
+        // ======================= publisher (one warp): the CTA's column partial of every SUM segment =======================
         Sched it(P);
         Seg g;
         int segs = 0;
@@ -777,22 +837,17 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         const bool mine = c0 < RP;
         while (it.next(g)) {
             if (g.phase != kPhaseSum) break;              // SUM segments come first in the schedule
-            const int idx = g.side * BH + g.s;
-            int rb = __ldcg(P.robust + idx);              // stable once the segment's attempt has been reached
-            if (g.extra) {
-                int go = 0;
-                if (lane == 0) go = poll_ge(P.epoch + idx, P.T, sAbort, P.status) ? 1 + __ldcg(P.robust + idx) : 0;
-                go = __shfl_sync(0xffffffffu, go, 0);
-                if (go == 0) ok = false;
-                if (go == 1) continue;
-                rb = 1;
-            }
+            const int idx = g.side * BH + g.s, li = it.local(g);
+            int go = 0;
+            if (lane == 0) go = seg_state(li, idx, g.attempt);
+            go = __shfl_sync(0xffffffffu, go, 0);
+            if (go == 0) ok = false;
+            if (g.extra && go == 1) continue;
+            const int rb = go == 2;
             const int par = segs & 1;
             if (ok) ok = wwait(bar(bSegFull + par), (segs >> 1) & 1);
             ++segs;
             if (!ok) continue;
-            // the epilogue warps read robust after their own epoch wait; re-read it now that they have arrived
-            rb = __ldcg(P.robust + idx);
             float k0 = rb ? neg_inf() : 0.f, s0 = 0.f, k1 = k0, s1 = 0.f;
             if (mine) {
                 const float *src = sPart + ((par * 16) * 64 + c0) * 2;
@@ -805,66 +860,122 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(bSegEmpty + par));
-            if (mine)
-                __stcg(reinterpret_cast<float4 *>(P.part + (((size_t)idx * P.maxslots + g.slot) * RP + c0) * 2),
-                       make_float4(k0, s0, k1, s1));
-            __threadfence();
-            __syncwarp();
-            int last = 0;
-            if (lane == 0) {
-                __threadfence();
-                last = atomicAdd(P.ticket + idx, 1u) == (unsigned)g.nslots - 1u;
-            }
-            last = __shfl_sync(0xffffffffu, last, 0);
-            if (!last) continue;
-            // ---- last CTA of the (slice, side): merge every slot in slot order, update G
-            __threadfence();
-            k0 = k1 = rb ? neg_inf() : 0.f; s0 = s1 = 0.f;
             if (mine) {
-                const float *src = P.part + ((size_t)idx * P.maxslots * RP + c0) * 2;
-                for (int p0 = 0; p0 < g.nslots; p0 += 8) {
-                    float4 pr[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        pr[u] = make_float4(neg_inf(), 0.f, neg_inf(), 0.f);
-                        if (p0 + u < g.nslots) pr[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(p0 + u) * RP * 2));
-                    }
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        if (rb) { pair_merge(k0, s0, pr[u].x, pr[u].y); pair_merge(k1, s1, pr[u].z, pr[u].w); }
-                        else { s0 += pr[u].y; s1 += pr[u].w; }
-                    }
-                }
+                // two buffers by attempt parity: a CTA may publish attempt a+1 while a slower one still gathers attempt a
+                unsigned long long *dst = P.part + ((((size_t)(g.attempt & 1) * 2 * BH + idx) * P.maxslots + g.slot) * RP + c0) * 2;
+                st_tagged(dst, k0, s0, (unsigned)g.attempt + 1u);
+                st_tagged(dst + 2, k1, s1, (unsigned)g.attempt + 1u);
             }
+        }
+        __syncwarp();
+        if (lane == 0) { __threadfence_block(); *sPubDone = 1; }
+    } else {
+        // ======================= gatherer (one warp): all slots of a (slice, side) -> this CTA's copy of G =======================
+        Sched it(P);
+        Seg g;
+        bool ok = true;
+        const int c0 = 2 * lane;
+        const bool mine = c0 < RP;
+        while (it.next(g)) {
+            if (g.phase != kPhaseSum) break;
+            const int idx = g.side * BH + g.s, li = it.local(g);
+            const bool cached = li < kMaxLoc;
+            int go = 0;
+            if (lane == 0) go = seg_state(li, idx, g.attempt);
+            go = __shfl_sync(0xffffffffu, go, 0);
+            if (go == 0) ok = false;
+            if (g.extra && go == 1) continue;
+            if (!ok) continue;
+            const int rb = go == 2;
+            const unsigned tag = (unsigned)g.attempt + 1u;
+            float k0 = rb ? neg_inf() : 0.f, s0 = 0.f, k1 = k0, s1 = 0.f;
+            const unsigned long long *src = P.part + ((((size_t)(g.attempt & 1) * 2 * BH + idx) * P.maxslots) * RP + c0) * 2;
+            for (int p0 = 0; p0 < g.nslots && ok; p0 += 8) {
+                unsigned long long w[8][4];
+                uint64_t t0 = 0;
+                for (uint32_t tries = 0;; ++tries) {
+                    bool ready = true;
+                    if (mine) {
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if (p0 + u < g.nslots) {
+                                ld_tagged(src + (size_t)(p0 + u) * RP * 2, w[u][0], w[u][1]);
+                                ld_tagged(src + (size_t)(p0 + u) * RP * 2 + 2, w[u][2], w[u][3]);
+                            }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if (p0 + u < g.nslots)
+                                ready = ready && (unsigned)(w[u][0] >> 32) == tag && (unsigned)(w[u][1] >> 32) == tag &&
+                                        (unsigned)(w[u][2] >> 32) == tag && (unsigned)(w[u][3] >> 32) == tag;
+                    }
+                    if (__all_sync(0xffffffffu, ready)) break;
+                    bool giveup = *sAbort != 0;
+                    if ((tries & 7u) == 7u) {
+                        const uint64_t now = global_timer_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > kWaitLimitNs) giveup = true;
+                    }
+                    if (__any_sync(0xffffffffu, giveup)) {
+                        if (lane == 0) { *sAbort = 1; atomicOr(P.status, 4 /* LOT_DEV_TIMEOUT */); }
+                        ok = false;
+                        break;
+                    }
+                    __nanosleep(64);
+                }
+                if (!ok || !mine) continue;
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (p0 + u < g.nslots) {
+                        const float a0 = __uint_as_float((unsigned)w[u][0]), b0 = __uint_as_float((unsigned)w[u][1]);
+                        const float a1 = __uint_as_float((unsigned)w[u][2]), b1 = __uint_as_float((unsigned)w[u][3]);
+                        if (rb) { pair_merge(k0, s0, a0, b0); pair_merge(k1, s1, a1, b1); }
+                        else { s0 += b0; s1 += b1; }
+                    }
+            }
+            if (!ok) continue;
             bool bad = false;
             if (!rb && mine) {
                 if (c0 < P.r && !(s0 >= kPlainFloor && s0 <= 3.0e38f)) bad = true;
                 if (c0 + 1 < P.r && !(s1 >= kPlainFloor && s1 <= 3.0e38f)) bad = true;
             }
             const int fail = __any_sync(0xffffffffu, bad);
-            const int itn = __ldcg(P.iter + idx);
+            const int itn = cached ? sIter[li] : __ldcg(P.iter + idx);
             if (!fail && mine) {
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     const int col = c0 + u;
                     if (col < P.r) {
-                        float *gp = P.G + (size_t)idx * RP + col;
                         const float kk = u ? k1 : k0, ss = u ? s1 : s0;
-                        const float gn = __ldcg(gp) + lg2(__ldg(P.beta + g.h * P.r + col) * (float)g.nvalid) - (kk + lg2(ss));
-                        if (!isfinite(gn)) atomicOr(P.status, 1 /* LOT_DEV_NONFINITE */);
-                        __stcg(gp, gn);
-                        if (itn + 1 == P.T) P.g_nat[(size_t)idx * P.r + col] = gn * P.eps_ln2;
+                        const float gold = cached ? sGc[li * 64 + col] : __ldcg(P.G + (size_t)idx * RP + col);
+                        const float gn = gold + lg2(__ldg(P.beta + g.h * P.r + col) * (float)g.nvalid) - (kk + lg2(ss));
+                        if (cached) sGc[li * 64 + col] = gn;
+                        else __stcg(P.G + (size_t)idx * RP + col, gn);
+                        if (g.slot == 0) {
+                            if (!isfinite(gn)) atomicOr(P.status, 1 /* LOT_DEV_NONFINITE */);
+                            if (itn + 1 == P.T) P.g_nat[(size_t)idx * P.r + col] = gn * P.eps_ln2;
+                        }
                     }
                 }
-                __threadfence();
             }
-            __syncwarp();
-            if (lane == 0) {
-                __stcg(P.ticket + idx, 0u);
-                if (fail) __stcg(P.robust + idx, 1);
+            if (cached) {
+                __threadfence_block();
+                __syncwarp();
+                if (lane == 0) {
+                    if (fail) sRobust[li] = 1;
+                    else sIter[li] = itn + 1;
+                    __threadfence_block();
+                    sDone[li] = g.attempt + 1;
+                }
+            } else {
+                // beyond the cache the state lives in global memory; every sharing CTA writes the same values
                 __threadfence();
-                if (!fail) st_release(P.iter + idx, itn + 1);
-                st_release(P.epoch + idx, g.attempt + 1);
+                __syncwarp();
+                if (lane == 0) {
+                    if (fail) __stcg(P.robust + idx, 1);
+                    __threadfence();
+                    if (!fail) st_release(P.iter + idx, itn + 1);
+                    st_release(P.epoch + idx, g.attempt + 1);
+                }
             }
         }
     }
@@ -979,7 +1090,6 @@ FusedLayout fused_layout(int B, int H, int n, int d, int r)
     size_t o = 0;
     L.status = o; o += 256;
     L.G = o; o += up256((size_t)2 * BH * RP * 4);
-    L.ticket = o; o += up256((size_t)2 * BH * 4);
     L.epoch = o; o += up256((size_t)2 * BH * 4);
     L.iter = o; o += up256((size_t)2 * BH * 4);
     L.robust = o; o += up256((size_t)2 * BH * 4);
@@ -987,9 +1097,9 @@ FusedLayout fused_layout(int B, int H, int n, int d, int r)
     L.wdone = o; o += up256((size_t)BH * 4);
     L.gnat = o; o += up256((size_t)2 * BH * r * 4);
     L.Wb = o; o += up256((size_t)BH * 2 * d * 64 * 2);
+    L.part = o; o += up256((size_t)2 * 2 * BH * ms * RP * 2 * 8);
     L.head_end = o;
     L.zprep = o; o += up256((size_t)H * 2 * RP * d * 2);
-    L.part = o; o += up256((size_t)2 * BH * ms * RP * 2 * 4);
     L.wpart = o; o += up256((size_t)BH * ms * 128 * d * 4);
     L.total = o;
     return L;
@@ -1030,8 +1140,7 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
         return cudaErrorInvalidValue;
     P.beta = beta; P.key_len = key_len;
     P.G = reinterpret_cast<float *>(w + L.G);
-    P.part = reinterpret_cast<float *>(w + L.part);
-    P.ticket = reinterpret_cast<unsigned *>(w + L.ticket);
+    P.part = reinterpret_cast<unsigned long long *>(w + L.part);
     P.epoch = reinterpret_cast<int *>(w + L.epoch);
     P.iter = reinterpret_cast<int *>(w + L.iter);
     P.robust = reinterpret_cast<int *>(w + L.robust);
