@@ -83,46 +83,62 @@ struct alignas(64) FusedParams {
 // and key_len only).
 // ---------------------------------------------------------------------------------------
 struct Seg {
-    int phase, attempt, extra, s, side, b, h, nvalid, t0, t1, slot, nslots;
+    int phase, attempt, extra, s, side, b, h, nvalid, t0, t1, slot, nslots, li;
 };
 
+// The static part of a (slice, side) of this CTA: what does not change from pass to pass.
+__device__ __forceinline__ bool seg_static(const FusedParams &P, int u0, int u1, int s_lo, int s, int side, Seg &g)
+{
+    g.s = s; g.side = side; g.b = s / P.H; g.h = s % P.H;
+    g.li = (s - s_lo) * 2 + (side ? 0 : 1);         // index among this CTA's segments of one pass
+    g.nvalid = P.n;
+    if (side == 1 && P.key_len != nullptr) g.nvalid = min(max(__ldg(P.key_len + g.b), 0), P.n);
+    const int vt = (g.nvalid + kTileRows - 1) / kTileRows;
+    g.t0 = max(u0 - s * P.TPS, 0);
+    g.t1 = min(u1 - s * P.TPS, vt);
+    const int c_lo = (s * P.TPS) / P.q, c_hi = (s * P.TPS + vt - 1) / P.q;
+    g.slot = (int)blockIdx.x - c_lo;
+    g.nslots = c_hi - c_lo + 1;
+    return g.t0 < g.t1;
+}
+constexpr int kSegInts = 10;   // table entry: s, side, b, h, nvalid, t0, t1, slot, nslots, (unused)
+
+// Enumeration of (pass, segment).  With at most kMaxLoc segments per pass the static parts come from a table in
+// shared memory filled once per CTA (no integer division on the way); otherwise they are recomputed.
 struct Sched {
     const FusedParams &P;
-    int u0, u1, s_lo, s_hi, pass, s, side_idx;
-    __device__ explicit Sched(const FusedParams &p) : P(p)
+    const int *tab;
+    int u0, u1, s_lo, s_hi, nloc, pass, cur;
+    __device__ Sched(const FusedParams &p, const int *table) : P(p), tab(table)
     {
         const int NT = p.B * p.H * p.TPS;
         u0 = blockIdx.x * p.q;
         u1 = min(NT, u0 + p.q);
         s_lo = u0 / p.TPS;
         s_hi = (u1 - 1) / p.TPS;
+        nloc = 2 * (s_hi - s_lo + 1);
+        if (nloc > kMaxLoc) tab = nullptr;
         pass = p.T == 0 ? 1 : 0;       // passes 0..T-1 SUM, T spare SUM, T+1 WRED, T+2 OUT
-        s = s_lo;
-        side_idx = 0;
+        cur = 0;
     }
-    // index of the (slice, side) among this CTA's segments of one pass
-    __device__ int local(const Seg &g) const { return (g.s - s_lo) * 2 + (g.side ? 0 : 1); }
     __device__ bool next(Seg &g)
     {
         for (;;) {
             if (pass > P.T + 2) return false;
-            if (s > s_hi) { s = s_lo; side_idx = 0; ++pass; continue; }
+            if (cur >= nloc) { cur = 0; ++pass; continue; }
+            const int li = cur++;
+            const int side = (li & 1) ? 0 : 1;                 // key side first
             const int phase = pass <= P.T ? kPhaseSum : (pass == P.T + 1 ? kPhaseWred : kPhaseOut);
-            const int nsides = phase == kPhaseSum ? 2 : 1;
-            if (side_idx >= nsides) { side_idx = 0; ++s; continue; }
-            const int side = phase == kPhaseSum ? (side_idx == 0 ? 1 : 0) : (phase == kPhaseWred ? 1 : 0);
-            ++side_idx;
+            if ((phase == kPhaseWred && side == 0) || (phase == kPhaseOut && side == 1)) continue;
+            if (tab != nullptr) {
+                const int *e = tab + li * kSegInts;
+                if (e[5] >= e[6]) continue;
+                g.s = e[0]; g.side = e[1]; g.b = e[2]; g.h = e[3]; g.nvalid = e[4]; g.t0 = e[5]; g.t1 = e[6];
+                g.slot = e[7]; g.nslots = e[8]; g.li = li;
+            } else if (!seg_static(P, u0, u1, s_lo, s_lo + (li >> 1), side, g)) {
+                continue;
+            }
             g.phase = phase; g.attempt = pass; g.extra = (phase == kPhaseSum && pass == P.T);
-            g.s = s; g.side = side; g.b = s / P.H; g.h = s % P.H;
-            g.nvalid = P.n;
-            if (side == 1 && P.key_len != nullptr) g.nvalid = min(max(__ldg(P.key_len + g.b), 0), P.n);
-            const int vt = (g.nvalid + kTileRows - 1) / kTileRows;
-            g.t0 = max(u0 - s * P.TPS, 0);
-            g.t1 = min(u1 - s * P.TPS, vt);
-            if (g.t0 >= g.t1) continue;
-            const int c_lo = (s * P.TPS) / P.q, c_hi = (s * P.TPS + vt - 1) / P.q;
-            g.slot = (int)blockIdx.x - c_lo;
-            g.nslots = c_hi - c_lo + 1;
             return true;
         }
     }
@@ -144,7 +160,8 @@ struct Plan {
     static constexpr int offG = offMisc + 128;                 // float sG[4][64]
     static constexpr int offGc = offG + kGroups * 64 * 4;      // float sGc[kMaxLoc][64]: this CTA's copy of the potentials
     static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust [kMaxLoc]
-    static constexpr int total = offState + 3 * kMaxLoc * 4;
+    static constexpr int offSeg = offState + 3 * kMaxLoc * 4;  // int sSeg[kMaxLoc][kSegInts]: static parts of the segments
+    static constexpr int total = offSeg + kMaxLoc * kSegInts * 4;
     // float sPart[2][16][64][2], the per-warp column pairs of the SUM passes, lives in the first plan buffer
     // (free until the WRED pass; the epilogue waits for the publisher's last read before it writes a plan tile)
     static constexpr int offPart = offP;
@@ -281,6 +298,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     volatile int *sIter = sDone + kMaxLoc;
     volatile int *sRobust = sIter + kMaxLoc;
     volatile int *sPubDone = reinterpret_cast<volatile int *>(smem + PL::offMisc + 12);
+    int *sSeg = reinterpret_cast<int *>(smem + PL::offSeg);
     // Wait until `need` attempts of local segment li (global index idx) are complete: 0 = gave up, else 1 + robust flag
     auto seg_state = [&](int li, int idx, int need) -> int {
         if (li < kMaxLoc) return spin_ge(sDone + li, need, sAbort, P.status) ? 1 + sRobust[li] : 0;
@@ -315,6 +333,20 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     if (warp == 1) { tmem_alloc(smem_u32(sTmem), PL::tmem_cols); tmem_relinquish(); }
     for (int i = threadIdx.x; i < kMaxLoc * 64; i += kThreads) sGc[i] = 0.f;
     if (threadIdx.x < 3 * kMaxLoc) sDone[threadIdx.x] = 0;
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + kMaxLoc) {
+        // segment table: one thread per (slice, side) of this CTA
+        const int li = threadIdx.x - 64;
+        const int NT = P.B * P.H * P.TPS, u0 = blockIdx.x * P.q, u1 = min(NT, u0 + P.q);
+        const int s_lo = u0 / P.TPS, s_hi = (u1 - 1) / P.TPS;
+        int *e = sSeg + li * kSegInts;
+        e[5] = 0; e[6] = 0;
+        if (li < 2 * (s_hi - s_lo + 1)) {
+            Seg g;
+            seg_static(P, u0, u1, s_lo, s_lo + (li >> 1), (li & 1) ? 0 : 1, g);
+            e[0] = g.s; e[1] = g.side; e[2] = g.b; e[3] = g.h; e[4] = g.nvalid; e[5] = g.t0; e[6] = g.t1;
+            e[7] = g.slot; e[8] = g.nslots;
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -327,14 +359,14 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     if (warp == 0) {
         // ======================= TMA producer (one lane) =======================
         if (lane == 0) {
-            Sched it(P);
+            Sched it(P, sSeg);
             Seg g;
             int kx = 0, ztag[2] = {-1, -1}, zuse[2] = {0, 0};
             bool ok = true;
             while (ok && it.next(g)) {
                 const int idx = g.side * BH + g.s;
                 if (g.extra) {
-                    const int go = seg_state(it.local(g), idx, P.T);
+                    const int go = seg_state(g.li, idx, P.T);
                     if (go == 0) { ok = false; break; }
                     if (go == 1) continue;
                 }
@@ -384,7 +416,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         // ======================= MMA issuer =======================
         // The whole warp runs the loop with warp-uniform values (so that descriptors and addresses can stay in
         // uniform registers); one elected lane issues the tcgen05 instructions.
-        Sched it(P);
+        Sched it(P, sSeg);
         Seg g;
         int k = 0, kx = 0, ztag[2] = {-1, -1}, zuse[2] = {0, 0}, segw = 0, sego = 0;
         int ka = 0, ko = 0;                   // tiles of the apply passes / of the OUT pass so far
@@ -438,7 +470,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             const int idx = g.side * BH + g.s;
             if (g.extra) {
                 int go = 0;
-                if (lane == 0) go = seg_state(it.local(g), idx, P.T);
+                if (lane == 0) go = seg_state(g.li, idx, P.T);
                 go = __shfl_sync(0xffffffffu, go, 0);
                 if (go == 0) { ok = false; break; }
                 if (go == 1) continue;
@@ -508,7 +540,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         const int rit = qd * 32 + lane;                                   // row-per-thread layout: row inside the tile
         const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
         float *myG = sG + grp * 64;
-        Sched it(P);
+        Sched it(P, sSeg);
         Seg g;
         int k = 0, ka = 0, ko = 0, segw = 0, sego = 0, segs = 0;
         bool ok = true;
@@ -518,7 +550,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             if (g.phase == kPhaseSum) {
                 // ================= SUM: quad layout, column sums in registers =================
                 // every warp waits by itself for the potential of this attempt
-                const int li = it.local(g);
+                const int li = g.li;
                 int go = 0;
                 if (lane == 0) go = seg_state(li, idx, g.attempt);
                 go = __shfl_sync(0xffffffffu, go, 0);
@@ -644,7 +676,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             }
 
             // ---- WRED / OUT: wait until the final potential (and W') of this slice is known here
-            const int li = it.local(g);
+            const int li = g.li;
             if (gtid == 0) {
                 bool w = spin_ge(sPubDone, 1, sAbort, P.status);          // plan buffers free of SUM partials
                 if (w) w = li < kMaxLoc ? spin_ge(sIter + li, P.T, sAbort, P.status) : poll_ge(P.iter + idx, P.T, sAbort, P.status);
@@ -829,7 +861,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         }
     } else if (warp == 18) {
         // ======================= publisher (one warp): the CTA's column partial of every SUM segment =======================
-        Sched it(P);
+        Sched it(P, sSeg);
         Seg g;
         int segs = 0;
         bool ok = true;
@@ -837,7 +869,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         const bool mine = c0 < RP;
         while (it.next(g)) {
             if (g.phase != kPhaseSum) break;              // SUM segments come first in the schedule
-            const int idx = g.side * BH + g.s, li = it.local(g);
+            const int idx = g.side * BH + g.s, li = g.li;
             int go = 0;
             if (lane == 0) go = seg_state(li, idx, g.attempt);
             go = __shfl_sync(0xffffffffu, go, 0);
@@ -871,14 +903,14 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         if (lane == 0) { __threadfence_block(); *sPubDone = 1; }
     } else {
         // ======================= gatherer (one warp): all slots of a (slice, side) -> this CTA's copy of G =======================
-        Sched it(P);
+        Sched it(P, sSeg);
         Seg g;
         bool ok = true;
         const int c0 = 2 * lane;
         const bool mine = c0 < RP;
         while (it.next(g)) {
             if (g.phase != kPhaseSum) break;
-            const int idx = g.side * BH + g.s, li = it.local(g);
+            const int idx = g.side * BH + g.s, li = g.li;
             const bool cached = li < kMaxLoc;
             int go = 0;
             if (lane == 0) go = seg_state(li, idx, g.attempt);

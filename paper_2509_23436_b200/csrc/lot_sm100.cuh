@@ -47,8 +47,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  `abort_flag` lives in shared memory; `status` is the global status word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+// Bounded wait.  `abort_flag` lives in shared memory; `status` is the global status word.  The common case
+// (phase already complete, or complete within the first suspended try) stays inline; the timed loop does not.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
     uint64_t t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -63,6 +64,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     atomicOr(status, 4 /* LOT_DEV_TIMEOUT */);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status);
 }
 
 __device__ __forceinline__ void fence_barrier_init()
