@@ -73,7 +73,8 @@ struct alignas(64) FusedParams {
     int *status;
     int B, H, n, r, T;
     int TPS;                     // tiles per slice = ceil(n / 128)
-    int q;                       // tiles per CTA and side
+    int q;                       // tiles per CTA and side (contiguous mapping)
+    int cps;                     // > 0: aligned mapping, this many CTAs per slice, none spanning two slices
     int maxslots;
     float eps_ln2;
 };
@@ -86,6 +87,31 @@ struct Seg {
     int phase, attempt, extra, s, side, b, h, nvalid, t0, t1, slot, nslots, li;
 };
 
+// Tile range [u0, u1) of a CTA in the slice-major tile list.  Aligned mapping: cps CTAs split every slice evenly, so
+// that no CTA works on two slices; contiguous mapping: q tiles per CTA regardless of slice borders.
+__device__ __forceinline__ void cta_range(const FusedParams &P, int cta, int &u0, int &u1)
+{
+    if (P.cps > 0) {
+        const int s = cta / P.cps, j = cta % P.cps;
+        u0 = s * P.TPS + (j * P.TPS) / P.cps;
+        u1 = s * P.TPS + ((j + 1) * P.TPS) / P.cps;
+    } else {
+        u0 = cta * P.q;
+        u1 = min(P.B * P.H * P.TPS, u0 + P.q);
+    }
+}
+// First CTA and number of CTAs that hold valid tiles [0, vt) of slice s.
+__device__ __forceinline__ void slice_slots(const FusedParams &P, int s, int vt, int &c_lo, int &nslots)
+{
+    if (P.cps > 0) {
+        c_lo = s * P.cps;
+        nslots = min(P.cps, (vt * P.cps + P.TPS - 1) / P.TPS);
+    } else {
+        c_lo = (s * P.TPS) / P.q;
+        nslots = (s * P.TPS + vt - 1) / P.q - c_lo + 1;
+    }
+}
+
 // The static part of a (slice, side) of this CTA: what does not change from pass to pass.
 __device__ __forceinline__ bool seg_static(const FusedParams &P, int u0, int u1, int s_lo, int s, int side, Seg &g)
 {
@@ -96,9 +122,9 @@ __device__ __forceinline__ bool seg_static(const FusedParams &P, int u0, int u1,
     const int vt = (g.nvalid + kTileRows - 1) / kTileRows;
     g.t0 = max(u0 - s * P.TPS, 0);
     g.t1 = min(u1 - s * P.TPS, vt);
-    const int c_lo = (s * P.TPS) / P.q, c_hi = (s * P.TPS + vt - 1) / P.q;
+    int c_lo;
+    slice_slots(P, s, vt, c_lo, g.nslots);
     g.slot = (int)blockIdx.x - c_lo;
-    g.nslots = c_hi - c_lo + 1;
     return g.t0 < g.t1;
 }
 constexpr int kSegInts = 10;   // table entry: s, side, b, h, nvalid, t0, t1, slot, nslots, (unused)
@@ -111,9 +137,7 @@ struct Sched {
     int u0, u1, s_lo, s_hi, nloc, pass, cur;
     __device__ Sched(const FusedParams &p, const int *table) : P(p), tab(table)
     {
-        const int NT = p.B * p.H * p.TPS;
-        u0 = blockIdx.x * p.q;
-        u1 = min(NT, u0 + p.q);
+        cta_range(p, blockIdx.x, u0, u1);
         s_lo = u0 / p.TPS;
         s_hi = (u1 - 1) / p.TPS;
         nloc = 2 * (s_hi - s_lo + 1);
@@ -336,7 +360,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     if (threadIdx.x >= 64 && threadIdx.x < 64 + kMaxLoc) {
         // segment table: one thread per (slice, side) of this CTA
         const int li = threadIdx.x - 64;
-        const int NT = P.B * P.H * P.TPS, u0 = blockIdx.x * P.q, u1 = min(NT, u0 + P.q);
+        int u0, u1;
+        cta_range(P, blockIdx.x, u0, u1);
         const int s_lo = u0 / P.TPS, s_hi = (u1 - 1) / P.TPS;
         int *e = sSeg + li * kSegInts;
         e[5] = 0; e[6] = 0;
@@ -1100,11 +1125,22 @@ bool fused_supported(int dtype, int d, int r)
     return dtype == 1 && d == fused::kDK && r >= 1 && r <= 64;
 }
 
-void fused_geometry(int B, int H, int n, int *q, int *ctas, int *maxslots)
+void fused_geometry(int B, int H, int n, int *q, int *ctas, int *maxslots, int *cps)
 {
     const int TPS = (n + 127) / 128;
-    const long long NT = (long long)B * H * TPS;
+    const long long BH = (long long)B * H, NT = BH * TPS;
     const int sms = fused::num_sms();
+    // aligned mapping when whole groups of CTAs per slice fill (nearly) all SMs: every CTA then has one
+    // (slice, side) per side and pass, and the CTAs of a slice stay in step
+    const int c = BH <= sms ? (int)(sms / BH) : 0;
+    if (c >= 1 && TPS >= c && BH * c * 100 >= 85ll * sms) {
+        *cps = c;
+        *q = (TPS + c - 1) / c;
+        *ctas = (int)(BH * c);
+        *maxslots = c;
+        return;
+    }
+    *cps = 0;
     int qq = (int)((NT + sms - 1) / sms);
     if (qq < 1) qq = 1;
     *q = qq;
@@ -1117,8 +1153,8 @@ FusedLayout fused_layout(int B, int H, int n, int d, int r)
     using fused::up256;
     FusedLayout L;
     const int BH = B * H, RP = fused::pad_r(r);
-    int q, ctas, ms;
-    fused_geometry(B, H, n, &q, &ctas, &ms);
+    int q, ctas, ms, cps;
+    fused_geometry(B, H, n, &q, &ctas, &ms, &cps);
     size_t o = 0;
     L.status = o; o += 256;
     L.G = o; o += up256((size_t)2 * BH * RP * 4);
@@ -1186,7 +1222,7 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
     P.B = B; P.H = H; P.n = n; P.r = r; P.T = iters;
     P.TPS = (n + 127) / 128;
     int ctas;
-    fused_geometry(B, H, n, &P.q, &ctas, &P.maxslots);
+    fused_geometry(B, H, n, &P.q, &ctas, &P.maxslots, &P.cps);
     P.eps_ln2 = (float)((double)eps * 0.6931471805599453);
 
     const float scale = (float)(1.4426950408889634 / (double)eps);

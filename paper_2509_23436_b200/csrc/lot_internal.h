@@ -67,7 +67,7 @@ struct FusedLayout {
     size_t status, G, epoch, iter, robust, wticket, wdone, gnat, Wb, head_end, zprep, part, wpart, total;
 };
 bool fused_supported(int dtype, int d, int r);
-void fused_geometry(int B, int H, int n, int *q, int *ctas, int *maxslots);
+void fused_geometry(int B, int H, int n, int *q, int *ctas, int *maxslots, int *cps);
 FusedLayout fused_layout(int B, int H, int n, int d, int r);
 cudaError_t fused_attention(const void *q, const void *k, const void *v, const float *z, const float *beta,
                             const int32_t *key_len, int B, int H, int n, int d, int r, float eps, int iters,
