@@ -15,9 +15,9 @@
 // tensor cores, W' = W / beta) and the OUT pass (query side: closing token update,
 // out = softmax-rows x W' on tensor cores).
 //
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-17 four epilogue
-// groups of 128 threads (tile k goes to group k % 4 and TMEM accumulator k % 4), warp 18 the
-// publisher, warp 19 the gatherer.  Producer and MMA issuer never depend on G, so they run
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 4-15 three epilogue
+// groups of 128 threads (tile k goes to group and TMEM accumulator k % 3), warp 2 the
+// publisher, warp 3 the gatherer.  Producer and MMA issuer never depend on G, so they run
 // ahead across pass boundaries; only the epilogue warps wait, per segment, for the potential of
 // that attempt.
 //
@@ -44,9 +44,11 @@ namespace fused {
 using namespace sm100;
 
 constexpr int kPhaseSum = 0, kPhaseWred = 1, kPhaseOut = 2;
-constexpr int kGroups = 4;
+constexpr int kGroups = 3;                        // epilogue groups of four warps (one per TMEM lane quarter)
+constexpr int kEpiWarps = kGroups * 4;
+constexpr int kWGroups = kGroups == 4 ? 4 : 2;    // groups that read the W accumulator out (64 / kWGroups columns each)
 constexpr int kEpiThreads = kGroups * 128;
-constexpr int kThreads = 64 + kEpiThreads + 64;
+constexpr int kThreads = 128 + kEpiThreads;        // warps 0-3: producer, MMA issuer, publisher, gatherer; then the epilogue
 constexpr int kMaxLoc = 16;                      // (slice, side) states of a CTA cached in shared memory
 constexpr int kTileRows = 128;
 constexpr int kDK = 64;                          // head dimension of this path
@@ -181,12 +183,12 @@ struct Plan {
     static constexpr int offW = offP + 2 * PBYTES;
     static constexpr int offBar = offW + WBYTES;               // 64 mbarriers
     static constexpr int offMisc = offBar + 64 * 8;            // abort flag, TMEM base, flags
-    static constexpr int offG = offMisc + 128;                 // float sG[4][64]
+    static constexpr int offG = offMisc + 128;                 // float sG[kGroups][64]
     static constexpr int offGc = offG + kGroups * 64 * 4;      // float sGc[kMaxLoc][64]: this CTA's copy of the potentials
     static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust [kMaxLoc]
     static constexpr int offSeg = offState + 3 * kMaxLoc * 4;  // int sSeg[kMaxLoc][kSegInts]: static parts of the segments
     static constexpr int total = offSeg + kMaxLoc * kSegInts * 4;
-    // float sPart[2][16][64][2], the per-warp column pairs of the SUM passes, lives in the first plan buffer
+    // float sPart[2][kEpiWarps][64][2], the per-warp column pairs of the SUM passes, lives in the first plan buffer
     // (free until the WRED pass; the epilogue waits for the publisher's last read before it writes a plan tile)
     static constexpr int offPart = offP;
     static constexpr int dyn_bytes = total + 1024;             // slack for 1024-byte alignment
@@ -346,9 +348,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             mbar_init(bar(bOFull + i), 1); mbar_init(bar(bOEmpty + i), 4);
         }
         for (int i = 0; i < kGroups; ++i) { mbar_init(bar(bAccFull + i), 1); mbar_init(bar(bAccEmpty + i), 4); }
-        mbar_init(bar(bWFull), 1); mbar_init(bar(bWEmpty), 16);
-        mbar_init(bar(bWqFull), 16); mbar_init(bar(bWqEmpty), 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(bSegFull + i), 16); mbar_init(bar(bSegEmpty + i), 1); }
+        mbar_init(bar(bWFull), 1); mbar_init(bar(bWEmpty), kEpiWarps);
+        mbar_init(bar(bWqFull), kEpiWarps); mbar_init(bar(bWqEmpty), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(bSegFull + i), kEpiWarps); mbar_init(bar(bSegEmpty + i), 1); }
         *sAbort = 0;
         *sPubDone = 0;
         fence_barrier_init();
@@ -357,9 +359,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     if (warp == 1) { tmem_alloc(smem_u32(sTmem), PL::tmem_cols); tmem_relinquish(); }
     for (int i = threadIdx.x; i < kMaxLoc * 64; i += kThreads) sGc[i] = 0.f;
     if (threadIdx.x < 3 * kMaxLoc) sDone[threadIdx.x] = 0;
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + kMaxLoc) {
+    if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxLoc) {
         // segment table: one thread per (slice, side) of this CTA
-        const int li = threadIdx.x - 64;
+        const int li = threadIdx.x - 128;
         int u0, u1;
         cta_range(P, blockIdx.x, u0, u1);
         const int s_lo = u0 / P.TPS, s_hi = (u1 - 1) / P.TPS;
@@ -381,6 +383,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     constexpr uint32_t idesc_w = make_idesc_bf16(128, DK, 1, 1);
     constexpr uint32_t idesc_o = make_idesc_bf16(128, DK, 0, 0);
 
+    // The four service warps need few registers; give what they release to the sixteen epilogue warps.
+    if (warp < 4) {
     if (warp == 0) {
         // ======================= TMA producer (one lane) =======================
         if (lane == 0) {
@@ -444,6 +448,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         Sched it(P, sSeg);
         Seg g;
         int k = 0, kx = 0, ztag[2] = {-1, -1}, zuse[2] = {0, 0}, segw = 0, sego = 0;
+        int gk = 0;                           // group of tile k, and per-group tile-count parities
+        uint32_t gpar = 0;
         int ka = 0, ko = 0;                   // tiles of the apply passes / of the OUT pass so far
         bool ok = true, w_open = false;
         int pend_k = -1, pend_o = 0, pend_first = 0, pend_vs = 0, pend_phase = 0;   // apply MMA still to be issued
@@ -526,10 +532,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             }
             const uint32_t za = dK_lo + ((PL::offZ + zs * PL::ZBYTES) >> 4);
             for (int t = g.t0; t < g.t1 && ok; ++t, ++k) {
-                const int grp = k & 3, j = k >> 2;
+                const int grp = gk;                         // tile k goes to group k % kGroups
+                const uint32_t gbit = (gpar >> grp) & 1;    // parity of this group's tile count
+                gpar ^= 1u << grp;
+                gk = gk + 1 == kGroups ? 0 : gk + 1;
                 const int st = kx % kStages, ph = (kx / kStages) & 1;
                 ok = wwait(bar(bXFull + st), ph);
-                if (ok) ok = wwait(bar(bAccEmpty + grp), (j & 1) ^ 1);
+                if (ok) ok = wwait(bar(bAccEmpty + grp), gbit ^ 1);
                 tc_fence_after();
                 const uint32_t xa = dK_lo + ((PL::offX + st * kStageBytes) >> 4);
                 const uint32_t dcol = tm + grp * RP;
@@ -557,10 +566,162 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         if (pend_k >= 0 && ok) issue_apply();
         if (w_open && ok && elect_one()) umma_commit(bar(bWFull));
         __syncwarp();
-    } else if (warp < 18) {
-        // ======================= epilogue (16 warps, 4 groups) =======================
-        const int ew = warp - 2, grp = ew >> 2, w4 = ew & 3, qd = warp & 3;
-        const int etid = threadIdx.x - 64, gtid = w4 * 32 + lane;
+    } else if (warp == 2) {
+        // ======================= publisher (one warp): the CTA's column partial of every SUM segment =======================
+        Sched it(P, sSeg);
+        Seg g;
+        int segs = 0;
+        bool ok = true;
+        const int c0 = 2 * lane;                          // this lane's two columns (lanes with c0 >= RP idle)
+        const bool mine = c0 < RP;
+        while (it.next(g)) {
+            if (g.phase != kPhaseSum) break;              // SUM segments come first in the schedule
+            const int idx = g.side * BH + g.s, li = g.li;
+            int go = 0;
+            if (lane == 0) go = seg_state(li, idx, g.attempt);
+            go = __shfl_sync(0xffffffffu, go, 0);
+            if (go == 0) ok = false;
+            if (g.extra && go == 1) continue;
+            const int rb = go == 2;
+            const int par = segs & 1;
+            if (ok) ok = wwait(bar(bSegFull + par), (segs >> 1) & 1);
+            ++segs;
+            if (!ok) continue;
+            float k0 = rb ? neg_inf() : 0.f, s0 = 0.f, k1 = k0, s1 = 0.f;
+            if (mine) {
+                const float *src = sPart + ((par * kEpiWarps) * 64 + c0) * 2;
+#pragma unroll
+                for (int w = 0; w < kEpiWarps; ++w) {
+                    const float4 pr = *reinterpret_cast<const float4 *>(src + w * 128);
+                    if (rb) { pair_merge(k0, s0, pr.x, pr.y); pair_merge(k1, s1, pr.z, pr.w); }
+                    else { s0 += pr.y; s1 += pr.w; }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(bSegEmpty + par));
+            if (mine) {
+                // two buffers by attempt parity: a CTA may publish attempt a+1 while a slower one still gathers attempt a
+                unsigned long long *dst = P.part + ((((size_t)(g.attempt & 1) * 2 * BH + idx) * P.maxslots + g.slot) * RP + c0) * 2;
+                st_tagged(dst, k0, s0, (unsigned)g.attempt + 1u);
+                st_tagged(dst + 2, k1, s1, (unsigned)g.attempt + 1u);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) { __threadfence_block(); *sPubDone = 1; }
+    } else {
+        // ======================= gatherer (one warp): all slots of a (slice, side) -> this CTA's copy of G =======================
+        Sched it(P, sSeg);
+        Seg g;
+        bool ok = true;
+        const int c0 = 2 * lane;
+        const bool mine = c0 < RP;
+        while (it.next(g)) {
+            if (g.phase != kPhaseSum) break;
+            const int idx = g.side * BH + g.s, li = g.li;
+            const bool cached = li < kMaxLoc;
+            int go = 0;
+            if (lane == 0) go = seg_state(li, idx, g.attempt);
+            go = __shfl_sync(0xffffffffu, go, 0);
+            if (go == 0) ok = false;
+            if (g.extra && go == 1) continue;
+            if (!ok) continue;
+            const int rb = go == 2;
+            const unsigned tag = (unsigned)g.attempt + 1u;
+            float k0 = rb ? neg_inf() : 0.f, s0 = 0.f, k1 = k0, s1 = 0.f;
+            const unsigned long long *src = P.part + ((((size_t)(g.attempt & 1) * 2 * BH + idx) * P.maxslots) * RP + c0) * 2;
+            for (int p0 = 0; p0 < g.nslots && ok; p0 += 4) {
+                unsigned long long w[4][4];
+                uint64_t t0 = 0;
+                for (uint32_t tries = 0;; ++tries) {
+                    bool ready = true;
+                    if (mine) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (p0 + u < g.nslots) {
+                                ld_tagged(src + (size_t)(p0 + u) * RP * 2, w[u][0], w[u][1]);
+                                ld_tagged(src + (size_t)(p0 + u) * RP * 2 + 2, w[u][2], w[u][3]);
+                            }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (p0 + u < g.nslots)
+                                ready = ready && (unsigned)(w[u][0] >> 32) == tag && (unsigned)(w[u][1] >> 32) == tag &&
+                                        (unsigned)(w[u][2] >> 32) == tag && (unsigned)(w[u][3] >> 32) == tag;
+                    }
+                    if (__all_sync(0xffffffffu, ready)) break;
+                    bool giveup = *sAbort != 0;
+                    if ((tries & 7u) == 7u) {
+                        const uint64_t now = global_timer_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > kWaitLimitNs) giveup = true;
+                    }
+                    if (__any_sync(0xffffffffu, giveup)) {
+                        if (lane == 0) { *sAbort = 1; atomicOr(P.status, 4 /* LOT_DEV_TIMEOUT */); }
+                        ok = false;
+                        break;
+                    }
+                    __nanosleep(64);
+                }
+                if (!ok || !mine) continue;
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (p0 + u < g.nslots) {
+                        const float a0 = __uint_as_float((unsigned)w[u][0]), b0 = __uint_as_float((unsigned)w[u][1]);
+                        const float a1 = __uint_as_float((unsigned)w[u][2]), b1 = __uint_as_float((unsigned)w[u][3]);
+                        if (rb) { pair_merge(k0, s0, a0, b0); pair_merge(k1, s1, a1, b1); }
+                        else { s0 += b0; s1 += b1; }
+                    }
+            }
+            if (!ok) continue;
+            bool bad = false;
+            if (!rb && mine) {
+                if (c0 < P.r && !(s0 >= kPlainFloor && s0 <= 3.0e38f)) bad = true;
+                if (c0 + 1 < P.r && !(s1 >= kPlainFloor && s1 <= 3.0e38f)) bad = true;
+            }
+            const int fail = __any_sync(0xffffffffu, bad);
+            const int itn = cached ? sIter[li] : __ldcg(P.iter + idx);
+            if (!fail && mine) {
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int col = c0 + u;
+                    if (col < P.r) {
+                        const float kk = u ? k1 : k0, ss = u ? s1 : s0;
+                        const float gold = cached ? sGc[li * 64 + col] : __ldcg(P.G + (size_t)idx * RP + col);
+                        const float gn = gold + lg2(__ldg(P.beta + g.h * P.r + col) * (float)g.nvalid) - (kk + lg2(ss));
+                        if (cached) sGc[li * 64 + col] = gn;
+                        else __stcg(P.G + (size_t)idx * RP + col, gn);
+                        if (g.slot == 0) {
+                            if (!isfinite(gn)) atomicOr(P.status, 1 /* LOT_DEV_NONFINITE */);
+                            if (itn + 1 == P.T) P.g_nat[(size_t)idx * P.r + col] = gn * P.eps_ln2;
+                        }
+                    }
+                }
+            }
+            if (cached) {
+                __threadfence_block();
+                __syncwarp();
+                if (lane == 0) {
+                    if (fail) sRobust[li] = 1;
+                    else sIter[li] = itn + 1;
+                    __threadfence_block();
+                    sDone[li] = g.attempt + 1;
+                }
+            } else {
+                // beyond the cache the state lives in global memory; every sharing CTA writes the same values
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) {
+                    if (fail) __stcg(P.robust + idx, 1);
+                    __threadfence();
+                    if (!fail) st_release(P.iter + idx, itn + 1);
+                    st_release(P.epoch + idx, g.attempt + 1);
+                }
+            }
+        }
+    }
+    } else {
+        // ======================= epilogue (kGroups groups of four warps) =======================
+        const int ew = warp - 4, grp = ew >> 2, w4 = ew & 3, qd = warp & 3;
+        const int etid = threadIdx.x - 128, gtid = w4 * 32 + lane;
         const int rq = lane >> 2, cq = lane & 3;                          // quad layout: row and column quarter
         const int rit = qd * 32 + lane;                                   // row-per-thread layout: row inside the tile
         const uint32_t lane_addr = tmem_base + ((uint32_t)(qd * 32) << 16);
@@ -568,6 +729,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         Sched it(P, sSeg);
         Seg g;
         int k = 0, ka = 0, ko = 0, segw = 0, sego = 0, segs = 0;
+        int gk = 0;                           // group of tile k
+        uint32_t mypar = 0;                   // parity of the number of tiles this group has taken
         bool ok = true;
 
         while (it.next(g)) {
@@ -582,7 +745,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 if (go == 0) ok = false;
                 const int rb = go == 2;
                 if (g.extra && go == 1) continue;                       // this segment needed no repeat
-                float *dstp = sPart + (((segs & 1) * 16 + ew) * 64) * 2;
+                float *dstp = sPart + (((segs & 1) * kEpiWarps + ew) * 64) * 2;
                 const uint32_t par_empty = ((segs >> 1) & 1) ^ 1;
                 const int par = segs & 1;
                 ++segs;
@@ -598,9 +761,11 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         if (RB) kap[ci] = neg_inf();
                     }
                     for (int t = g.t0; t < g.t1; ++t, ++k) {
-                        if ((k & 3) != grp) continue;
-                        const int j = k >> 2;
-                        if (ok) ok = wwait(bar(bAccFull + grp), j & 1);
+                        const bool mine = gk == grp;
+                        gk = gk + 1 == kGroups ? 0 : gk + 1;
+                        if (!mine) continue;
+                        if (ok) ok = wwait(bar(bAccFull + grp), mypar);
+                        mypar ^= 1u;
                         if (!ok) continue;
                         tc_fence_after();
 #pragma unroll
@@ -721,9 +886,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 // stage W'^T (hi, lo) of this slice as the B operand: 128-byte rows, 16-byte chunks xor row%8
                 if (sego > 0 && ok) ok = wwait(bar(bWqEmpty), (sego - 1) & 1);
                 const uint4 *src = reinterpret_cast<const uint4 *>(P.Wb + (size_t)g.s * 2 * DK * 64);
-#pragma unroll
-                for (int rep = 0; rep < 2; ++rep) {
-                    const int c = etid + rep * kEpiThreads;          // 1024 chunks of 16 bytes
+                for (int c = etid; c < 1024; c += kEpiThreads) {       // 1024 chunks of 16 bytes
                     const int part = c >> 9, row = (c >> 3) & 63, ch = c & 7;
                     const uint4 val = __ldcg(src + c);
                     *reinterpret_cast<uint4 *>(smem + PL::offW + part * (DK * 128) + row * 128 + ((ch ^ (row & 7)) * 16)) = val;
@@ -739,9 +902,11 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 const int pb = ka & 1, pj = ka >> 1, ob = ko & 1, oj = ko >> 1;
                 ++ka;
                 if (g.phase == kPhaseOut) ++ko;
-                if ((k & 3) != grp) continue;
-                const int j = k >> 2;
-                if (ok) ok = wwait(bar(bAccFull + grp), j & 1);
+                const bool mine = gk == grp;
+                gk = gk + 1 == kGroups ? 0 : gk + 1;
+                if (!mine) continue;
+                if (ok) ok = wwait(bar(bAccFull + grp), mypar);
+                mypar ^= 1u;
                 if (!ok) continue;
                 tc_fence_after();
                 const int row = t * kTileRows + rit;
@@ -818,18 +983,23 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 // ---- W accumulator of this segment: warp (qd, grp) takes its 32 lanes x 16 channels
                 if (ok) ok = wwait(bar(bWFull), segw & 1);
                 if (ok) {
+                    constexpr int WC = DK / kWGroups;              // channels per reading group
                     tc_fence_after();
-                    float wv[16];
-                    tmem_ld16(lane_addr + PL::colW + grp * 16, wv);
-                    tmem_wait_ld();
+                    float wv[WC];
+                    if (grp < kWGroups) {
+                        tmem_ld<WC>(lane_addr + PL::colW + grp * WC, wv);
+                        tmem_wait_ld();
+                    }
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(bWEmpty));
-                    float *dst = P.wpart + (((size_t)g.s * P.maxslots + g.slot) * 128 + rit) * DK + grp * 16;
+                    if (grp < kWGroups) {
+                        float *dst = P.wpart + (((size_t)g.s * P.maxslots + g.slot) * 128 + rit) * DK + grp * WC;
 #pragma unroll
-                    for (int c = 0; c < 16; c += 4)
-                        __stcg(reinterpret_cast<float4 *>(dst + c), make_float4(wv[c], wv[c + 1], wv[c + 2], wv[c + 3]));
-                    __threadfence();
+                        for (int c = 0; c < WC; c += 4)
+                            __stcg(reinterpret_cast<float4 *>(dst + c), make_float4(wv[c], wv[c + 1], wv[c + 2], wv[c + 3]));
+                        __threadfence();
+                    }
                 }
                 ++segw;
                 named_bar_sync(5, kEpiThreads);
@@ -881,157 +1051,6 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         __threadfence();
                         st_release(P.wdone + g.s, 1);
                     }
-                }
-            }
-        }
-    } else if (warp == 18) {
-        // ======================= publisher (one warp): the CTA's column partial of every SUM segment =======================
-        Sched it(P, sSeg);
-        Seg g;
-        int segs = 0;
-        bool ok = true;
-        const int c0 = 2 * lane;                          // this lane's two columns (lanes with c0 >= RP idle)
-        const bool mine = c0 < RP;
-        while (it.next(g)) {
-            if (g.phase != kPhaseSum) break;              // SUM segments come first in the schedule
-            const int idx = g.side * BH + g.s, li = g.li;
-            int go = 0;
-            if (lane == 0) go = seg_state(li, idx, g.attempt);
-            go = __shfl_sync(0xffffffffu, go, 0);
-            if (go == 0) ok = false;
-            if (g.extra && go == 1) continue;
-            const int rb = go == 2;
-            const int par = segs & 1;
-            if (ok) ok = wwait(bar(bSegFull + par), (segs >> 1) & 1);
-            ++segs;
-            if (!ok) continue;
-            float k0 = rb ? neg_inf() : 0.f, s0 = 0.f, k1 = k0, s1 = 0.f;
-            if (mine) {
-                const float *src = sPart + ((par * 16) * 64 + c0) * 2;
-#pragma unroll
-                for (int w = 0; w < 16; ++w) {
-                    const float4 pr = *reinterpret_cast<const float4 *>(src + w * 128);
-                    if (rb) { pair_merge(k0, s0, pr.x, pr.y); pair_merge(k1, s1, pr.z, pr.w); }
-                    else { s0 += pr.y; s1 += pr.w; }
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(bSegEmpty + par));
-            if (mine) {
-                // two buffers by attempt parity: a CTA may publish attempt a+1 while a slower one still gathers attempt a
-                unsigned long long *dst = P.part + ((((size_t)(g.attempt & 1) * 2 * BH + idx) * P.maxslots + g.slot) * RP + c0) * 2;
-                st_tagged(dst, k0, s0, (unsigned)g.attempt + 1u);
-                st_tagged(dst + 2, k1, s1, (unsigned)g.attempt + 1u);
-            }
-        }
-        __syncwarp();
-        if (lane == 0) { __threadfence_block(); *sPubDone = 1; }
-    } else {
-        // ======================= gatherer (one warp): all slots of a (slice, side) -> this CTA's copy of G =======================
-        Sched it(P, sSeg);
-        Seg g;
-        bool ok = true;
-        const int c0 = 2 * lane;
-        const bool mine = c0 < RP;
-        while (it.next(g)) {
-            if (g.phase != kPhaseSum) break;
-            const int idx = g.side * BH + g.s, li = g.li;
-            const bool cached = li < kMaxLoc;
-            int go = 0;
-            if (lane == 0) go = seg_state(li, idx, g.attempt);
-            go = __shfl_sync(0xffffffffu, go, 0);
-            if (go == 0) ok = false;
-            if (g.extra && go == 1) continue;
-            if (!ok) continue;
-            const int rb = go == 2;
-            const unsigned tag = (unsigned)g.attempt + 1u;
-            float k0 = rb ? neg_inf() : 0.f, s0 = 0.f, k1 = k0, s1 = 0.f;
-            const unsigned long long *src = P.part + ((((size_t)(g.attempt & 1) * 2 * BH + idx) * P.maxslots) * RP + c0) * 2;
-            for (int p0 = 0; p0 < g.nslots && ok; p0 += 8) {
-                unsigned long long w[8][4];
-                uint64_t t0 = 0;
-                for (uint32_t tries = 0;; ++tries) {
-                    bool ready = true;
-                    if (mine) {
-#pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            if (p0 + u < g.nslots) {
-                                ld_tagged(src + (size_t)(p0 + u) * RP * 2, w[u][0], w[u][1]);
-                                ld_tagged(src + (size_t)(p0 + u) * RP * 2 + 2, w[u][2], w[u][3]);
-                            }
-#pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            if (p0 + u < g.nslots)
-                                ready = ready && (unsigned)(w[u][0] >> 32) == tag && (unsigned)(w[u][1] >> 32) == tag &&
-                                        (unsigned)(w[u][2] >> 32) == tag && (unsigned)(w[u][3] >> 32) == tag;
-                    }
-                    if (__all_sync(0xffffffffu, ready)) break;
-                    bool giveup = *sAbort != 0;
-                    if ((tries & 7u) == 7u) {
-                        const uint64_t now = global_timer_ns();
-                        if (t0 == 0) t0 = now;
-                        else if (now - t0 > kWaitLimitNs) giveup = true;
-                    }
-                    if (__any_sync(0xffffffffu, giveup)) {
-                        if (lane == 0) { *sAbort = 1; atomicOr(P.status, 4 /* LOT_DEV_TIMEOUT */); }
-                        ok = false;
-                        break;
-                    }
-                    __nanosleep(64);
-                }
-                if (!ok || !mine) continue;
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (p0 + u < g.nslots) {
-                        const float a0 = __uint_as_float((unsigned)w[u][0]), b0 = __uint_as_float((unsigned)w[u][1]);
-                        const float a1 = __uint_as_float((unsigned)w[u][2]), b1 = __uint_as_float((unsigned)w[u][3]);
-                        if (rb) { pair_merge(k0, s0, a0, b0); pair_merge(k1, s1, a1, b1); }
-                        else { s0 += b0; s1 += b1; }
-                    }
-            }
-            if (!ok) continue;
-            bool bad = false;
-            if (!rb && mine) {
-                if (c0 < P.r && !(s0 >= kPlainFloor && s0 <= 3.0e38f)) bad = true;
-                if (c0 + 1 < P.r && !(s1 >= kPlainFloor && s1 <= 3.0e38f)) bad = true;
-            }
-            const int fail = __any_sync(0xffffffffu, bad);
-            const int itn = cached ? sIter[li] : __ldcg(P.iter + idx);
-            if (!fail && mine) {
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int col = c0 + u;
-                    if (col < P.r) {
-                        const float kk = u ? k1 : k0, ss = u ? s1 : s0;
-                        const float gold = cached ? sGc[li * 64 + col] : __ldcg(P.G + (size_t)idx * RP + col);
-                        const float gn = gold + lg2(__ldg(P.beta + g.h * P.r + col) * (float)g.nvalid) - (kk + lg2(ss));
-                        if (cached) sGc[li * 64 + col] = gn;
-                        else __stcg(P.G + (size_t)idx * RP + col, gn);
-                        if (g.slot == 0) {
-                            if (!isfinite(gn)) atomicOr(P.status, 1 /* LOT_DEV_NONFINITE */);
-                            if (itn + 1 == P.T) P.g_nat[(size_t)idx * P.r + col] = gn * P.eps_ln2;
-                        }
-                    }
-                }
-            }
-            if (cached) {
-                __threadfence_block();
-                __syncwarp();
-                if (lane == 0) {
-                    if (fail) sRobust[li] = 1;
-                    else sIter[li] = itn + 1;
-                    __threadfence_block();
-                    sDone[li] = g.attempt + 1;
-                }
-            } else {
-                // beyond the cache the state lives in global memory; every sharing CTA writes the same values
-                __threadfence();
-                __syncwarp();
-                if (lane == 0) {
-                    if (fail) __stcg(P.robust + idx, 1);
-                    __threadfence();
-                    if (!fail) st_release(P.iter + idx, itn + 1);
-                    st_release(P.epoch + idx, g.attempt + 1);
                 }
             }
         }
