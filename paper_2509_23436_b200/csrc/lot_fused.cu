@@ -898,10 +898,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             }
             named_bar_sync(1 + grp, 128);
 
+            // the tile loop is compiled once per pass kind, so that the other kind's work is not carried along
+            auto tiles = [&](auto wtag) {
+                constexpr bool WRED = decltype(wtag)::value;
             for (int t = g.t0; t < g.t1; ++t, ++k) {
                 const int pb = ka & 1, pj = ka >> 1, ob = ko & 1, oj = ko >> 1;
                 ++ka;
-                if (g.phase == kPhaseOut) ++ko;
+                if (!WRED) ++ko;
                 const bool mine = gk == grp;
                 gk = gk + 1 == kGroups ? 0 : gk + 1;
                 if (!mine) continue;
@@ -917,18 +920,30 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(bAccEmpty + grp));
-                float m = neg_inf();
+                // four independent chains for the row maximum and the row sum
+                float m4[4] = {neg_inf(), neg_inf(), neg_inf(), neg_inf()};
 #pragma unroll
-                for (int c = 0; c < RP; ++c) { v[c] += myG[c]; m = fmaxf(m, v[c]); }
-                float s = 0.f;
+                for (int c = 0; c < RP; c += 8) {
 #pragma unroll
-                for (int c = 0; c < RP; ++c) { v[c] = ex2(v[c] - m); s += v[c]; }
-                const float inv = __fdividef(1.f, s);
+                    for (int u = 0; u < 4; ++u) {
+                        v[c + 2 * u] += myG[c + 2 * u];
+                        v[c + 2 * u + 1] += myG[c + 2 * u + 1];
+                        m4[u] = max3(m4[u], v[c + 2 * u], v[c + 2 * u + 1]);
+                    }
+                }
+                const float m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+                float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int c = 0; c < RP; c += 4) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) { v[c + u] = ex2(v[c + u] - m); s4[u] += v[c + u]; }
+                }
+                const float inv = __fdividef(1.f, (s4[0] + s4[1]) + (s4[2] + s4[3]));
                 // ---- write the plan tile as an MMA operand
                 ok = wwait(bar(bPEmpty + pb), (pj & 1) ^ 1);
                 if (!ok) continue;
                 uint8_t *prow = smem + PL::offP + pb * PL::PBYTES + rit * 128;
-                const float w = g.phase == kPhaseWred ? (valid ? inv : 0.f) : 1.f;
+                const float w = WRED ? (valid ? inv : 0.f) : 1.f;
 #pragma unroll
                 for (int c8 = 0; c8 < 8; ++c8) {
                     uint32_t hi[4], lo[4];
@@ -943,13 +958,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     }
                     const int pc = (c8 ^ (rit & 7)) * 16;
                     *reinterpret_cast<uint4 *>(prow + pc) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                    if (g.phase == kPhaseWred)
+                    if (WRED)
                         *reinterpret_cast<uint4 *>(prow + kStageBytes + pc) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(bPFull + pb));
-                if (g.phase == kPhaseOut) {
+                if (!WRED) {
                     ok = wwait(bar(bOFull + ob), oj & 1);
                     if (!ok) continue;
                     tc_fence_after();
@@ -978,6 +993,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     }
                 }
             }
+            };
+            if (g.phase == kPhaseWred) tiles(std::true_type{});
+            else tiles(std::false_type{});
 
             if (g.phase == kPhaseWred) {
                 // ---- W accumulator of this segment: warp (qd, grp) takes its 32 lanes x 16 channels
@@ -1015,12 +1033,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     // 64 pivots x 64 channels, four channels per thread; slots in order, four slots of loads in flight
                     for (int e = etid; e < 64 * DK / 4; e += kEpiThreads) {
                         const int tt = e / (DK / 4), c = (e % (DK / 4)) * 4;
+                        const float bt = tt < P.r ? __ldg(P.beta + g.h * P.r + tt) : 1.f;   // issued with the partial loads
                         float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
                         const float *src0 = P.wpart + ((size_t)g.s * P.maxslots * 128) * DK + c;
-                        for (int sl0 = 0; sl0 < g.nslots; sl0 += 4) {
-                            float4 a[4], b[4];
+                        for (int sl0 = 0; sl0 < g.nslots; sl0 += 12) {
+                            float4 a[12], b[12];
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
+                            for (int u = 0; u < 12; ++u) {
                                 a[u] = b[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                                 if (sl0 + u < g.nslots) {
                                     const float *src = src0 + ((size_t)(sl0 + u) * 128) * DK;
@@ -1029,12 +1048,12 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                                 }
                             }
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
+                            for (int u = 0; u < 12; ++u) {
                                 sum.x += a[u].x + b[u].x; sum.y += a[u].y + b[u].y;
                                 sum.z += a[u].z + b[u].z; sum.w += a[u].w + b[u].w;
                             }
                         }
-                        const float sc = tt < P.r ? mass / __ldg(P.beta + g.h * P.r + tt) : 0.f;
+                        const float sc = tt < P.r ? mass / bt : 0.f;
                         const float wv[4] = {sum.x * sc, sum.y * sc, sum.z * sc, sum.w * sc};
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
