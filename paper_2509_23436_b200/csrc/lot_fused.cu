@@ -59,8 +59,11 @@ constexpr float kPlainFloor = 8.2718061e-25f;    // 2^-80: smallest column mass 
 struct alignas(64) FusedParams {
     CUtensorMap tmQ, tmK, tmV;   // [BH][n][64] bf16, box 64 x 128 x 1
     CUtensorMap tmZ;             // [2H][RP][64] bf16 (hi, lo of scaled pivots), box 64 x RP x 1
+    CUtensorMap tmKt;            // [2BH][npad][64] bf16 stored Gibbs kernel (r > 32 only), box 64 x 128 x 1
     const float *beta;           // [H][r]
     const int32_t *key_len;      // [B] or nullptr
+    __nv_bfloat16 *Kt;           // [2][BH][npad][64]: 2^(L_it - rowmax_i L), written by the first pass, or nullptr
+    int npad;                    // TPS * 128
     float *G;                    // [2][BH][RP] pivot potentials, base-2 units (side 0 = queries, 1 = keys)
     unsigned long long *part;    // [2 attempt parities][2][BH][maxslots][RP][2] tagged words per CTA slot: (kappa, tag), (S, tag)
     int *epoch;                  // [2][BH] attempts finished (used for segments beyond the shared-memory cache)
@@ -185,8 +188,8 @@ struct Plan {
     static constexpr int offMisc = offBar + 64 * 8;            // abort flag, TMEM base, flags
     static constexpr int offG = offMisc + 128;                 // float sG[kGroups][64]
     static constexpr int offGc = offG + kGroups * 64 * 4;      // float sGc[kMaxLoc][64]: this CTA's copy of the potentials
-    static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust [kMaxLoc]
-    static constexpr int offSeg = offState + 3 * kMaxLoc * 4;  // int sSeg[kMaxLoc][kSegInts]: static parts of the segments
+    static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust, sMode [kMaxLoc]
+    static constexpr int offSeg = offState + 4 * kMaxLoc * 4;  // int sSeg[kMaxLoc][kSegInts]: static parts of the segments
     static constexpr int total = offSeg + kMaxLoc * kSegInts * 4;
     // float sPart[2][kEpiWarps][64][2], the per-warp column pairs of the SUM passes, lives in the first plan buffer
     // (free until the WRED pass; the epilogue waits for the publisher's last read before it writes a plan tile)
@@ -323,11 +326,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     volatile int *sDone = reinterpret_cast<volatile int *>(smem + PL::offState);
     volatile int *sIter = sDone + kMaxLoc;
     volatile int *sRobust = sIter + kMaxLoc;
+    volatile int *sMode = sRobust + kMaxLoc;     // 1 = the next attempt reads the stored Gibbs kernel
     volatile int *sPubDone = reinterpret_cast<volatile int *>(smem + PL::offMisc + 12);
     int *sSeg = reinterpret_cast<int *>(smem + PL::offSeg);
-    // Wait until `need` attempts of local segment li (global index idx) are complete: 0 = gave up, else 1 + robust flag
+    // Wait until `need` attempts of local segment li (global index idx) are complete: 0 = gave up, else
+    // 1 + robust flag + 2 * (the attempt reads the stored Gibbs kernel)
     auto seg_state = [&](int li, int idx, int need) -> int {
-        if (li < kMaxLoc) return spin_ge(sDone + li, need, sAbort, P.status) ? 1 + sRobust[li] : 0;
+        if (li < kMaxLoc) return spin_ge(sDone + li, need, sAbort, P.status) ? 1 + sRobust[li] + 2 * sMode[li] : 0;
         return poll_ge(P.epoch + idx, need, sAbort, P.status) ? 1 + __ldcg(P.robust + idx) : 0;
     };
     auto bar = [&](int id) { return smem_u32(bars + id); };
@@ -355,10 +360,11 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         *sPubDone = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.tmQ); prefetch_tensormap(&P.tmK); prefetch_tensormap(&P.tmZ); prefetch_tensormap(&P.tmV);
+        if (P.Kt != nullptr) prefetch_tensormap(&P.tmKt);
     }
     if (warp == 1) { tmem_alloc(smem_u32(sTmem), PL::tmem_cols); tmem_relinquish(); }
     for (int i = threadIdx.x; i < kMaxLoc * 64; i += kThreads) sGc[i] = 0.f;
-    if (threadIdx.x < 3 * kMaxLoc) sDone[threadIdx.x] = 0;
+    if (threadIdx.x < 4 * kMaxLoc) sDone[threadIdx.x] = 0;
     if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxLoc) {
         // segment table: one thread per (slice, side) of this CTA
         const int li = threadIdx.x - 128;
@@ -394,10 +400,24 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             bool ok = true;
             while (ok && it.next(g)) {
                 const int idx = g.side * BH + g.s;
-                if (g.extra) {
-                    const int go = seg_state(g.li, idx, P.T);
+                bool resident = false;
+                if (g.phase == kPhaseSum && g.attempt > 0) {
+                    const int go = seg_state(g.li, idx, g.attempt);
                     if (go == 0) { ok = false; break; }
-                    if (go == 1) continue;
+                    if (g.extra && ((go - 1) & 1) == 0) continue;
+                    resident = (go - 1) >> 1;
+                }
+                if (resident) {
+                    // tiles of the stored Gibbs kernel instead of token tiles; no pivots, no MMA
+                    for (int t = g.t0; t < g.t1 && ok; ++t) {
+                        const int st = kx % kStages, ph = (kx / kStages) & 1;
+                        ok = mbar_wait(bar(bXEmpty + st), ph ^ 1, sAbort, P.status);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(bar(bXFull + st), kStageBytes);
+                        tma_load_3d(sbase + PL::offX + st * kStageBytes, &P.tmKt, bar(bXFull + st), 0, t * kTileRows, idx);
+                        ++kx;
+                    }
+                    continue;
                 }
                 const int zs = g.h & 1;
                 if (ztag[zs] != g.h) {
@@ -499,12 +519,17 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
 
         while (ok && it.next(g)) {
             const int idx = g.side * BH + g.s;
-            if (g.extra) {
+            if (g.phase == kPhaseSum && g.attempt > 0) {
                 int go = 0;
-                if (lane == 0) go = seg_state(g.li, idx, P.T);
+                if (lane == 0) go = seg_state(g.li, idx, g.attempt);
                 go = __shfl_sync(0xffffffffu, go, 0);
                 if (go == 0) { ok = false; break; }
-                if (go == 1) continue;
+                if (g.extra && ((go - 1) & 1) == 0) continue;
+                if ((go - 1) >> 1) {                     // the epilogue reads the stored Gibbs kernel: nothing to issue
+                    kx += g.t1 - g.t0;
+                    k += g.t1 - g.t0;
+                    continue;
+                }
             }
             if (pend_k >= 0) issue_apply();
             if (w_open) {                                                    // W of the previous WRED segment complete
@@ -581,8 +606,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             if (lane == 0) go = seg_state(li, idx, g.attempt);
             go = __shfl_sync(0xffffffffu, go, 0);
             if (go == 0) ok = false;
-            if (g.extra && go == 1) continue;
-            const int rb = go == 2;
+            if (g.extra && ((go - 1) & 1) == 0) continue;
+            const int rb = (go - 1) & 1;
             const int par = segs & 1;
             if (ok) ok = wwait(bar(bSegFull + par), (segs >> 1) & 1);
             ++segs;
@@ -623,9 +648,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             if (lane == 0) go = seg_state(li, idx, g.attempt);
             go = __shfl_sync(0xffffffffu, go, 0);
             if (go == 0) ok = false;
-            if (g.extra && go == 1) continue;
+            if (g.extra && ((go - 1) & 1) == 0) continue;
             if (!ok) continue;
-            const int rb = go == 2;
+            const int rb = (go - 1) & 1;
             const unsigned tag = (unsigned)g.attempt + 1u;
             float k0 = rb ? neg_inf() : 0.f, s0 = 0.f, k1 = k0, s1 = 0.f;
             const unsigned long long *src = P.part + ((((size_t)(g.attempt & 1) * 2 * BH + idx) * P.maxslots) * RP + c0) * 2;
@@ -696,10 +721,25 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     }
                 }
             }
+            // the next attempt may read the stored kernel if the potentials' spread keeps 2^(G - max G) well inside
+            // the float32 range (it decides how small a row sum can get)
+            float gmx = neg_inf(), gmn = -neg_inf();
+            if (RP == 64 && cached && !fail && mine) {
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    if (c0 + u < P.r) { const float gv = sGc[li * 64 + c0 + u]; gmx = fmaxf(gmx, gv); gmn = fminf(gmn, gv); }
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) {
+                gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, off));
+                gmn = fminf(gmn, __shfl_xor_sync(0xffffffffu, gmn, off));
+            }
+            const int next_resident = RP == 64 && cached && !fail && !rb && P.Kt != nullptr && (gmx - gmn) <= 64.f;
             if (cached) {
                 __threadfence_block();
                 __syncwarp();
                 if (lane == 0) {
+                    sMode[li] = next_resident;
                     if (fail) sRobust[li] = 1;
                     else sIter[li] = itn + 1;
                     __threadfence_block();
@@ -730,6 +770,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         Seg g;
         int k = 0, ka = 0, ko = 0, segw = 0, sego = 0, segs = 0;
         int gk = 0;                           // group of tile k
+        int kx = 0;                           // ring stage counter, as in the producer
         uint32_t mypar = 0;                   // parity of the number of tiles this group has taken
         bool ok = true;
 
@@ -743,12 +784,91 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 if (lane == 0) go = seg_state(li, idx, g.attempt);
                 go = __shfl_sync(0xffffffffu, go, 0);
                 if (go == 0) ok = false;
-                const int rb = go == 2;
-                if (g.extra && go == 1) continue;                       // this segment needed no repeat
+                const int rb = (go - 1) & 1, resident = go > 0 ? (go - 1) >> 1 : 0;
+                if (g.extra && rb == 0) continue;                       // this segment needed no repeat
                 float *dstp = sPart + (((segs & 1) * kEpiWarps + ew) * 64) * 2;
                 const uint32_t par_empty = ((segs >> 1) & 1) ^ 1;
                 const int par = segs & 1;
                 ++segs;
+
+                if constexpr (RP == 64) {
+                    if (resident) {
+                        // ---- stored-kernel pass: K~_it = 2^(L_it - max_t L_it) comes back as bf16 tiles; with
+                        // w_t = 2^(G_t - max G) the row sums are s_i = sum_t K~_it w_t and the column sums
+                        // w_t sum_i K~_it / s_i: two FMAs per entry, no exponential, no tensor-core work.
+                        // Thread = 4 rows (rq + 8 j of the warp's 32) x 16 consecutive columns (16 cq ..).
+                        float w[16], c[16];
+                        float gmax = neg_inf();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int col = cq * 16 + j;
+                            w[j] = col < P.r ? sGc[li * 64 + col] : neg_inf();
+                            gmax = fmaxf(gmax, w[j]);
+                            c[j] = 0.f;
+                        }
+                        gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
+                        gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) w[j] = ex2(w[j] - gmax);
+                        int lt = 0;
+                        for (int t = g.t0; t < g.t1; ++t, ++k, ++kx) {
+                            const bool mine = lt == grp;
+                            lt = lt + 1 == kGroups ? 0 : lt + 1;
+                            if (!mine) continue;
+                            const int stg = kx % kStages;
+                            if (ok) ok = wwait(bar(bXFull + stg), (kx / kStages) & 1);
+                            if (ok) {
+                                const uint8_t *tile = smem + PL::offX + stg * kStageBytes;
+#pragma unroll
+                                for (int jr = 0; jr < 4; ++jr) {
+                                    const int rin = w4 * 32 + jr * 8 + rq;           // row inside the tile
+                                    const uint4 a = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq) ^ (rin & 7)) * 16));
+                                    const uint4 b = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq + 1) ^ (rin & 7)) * 16));
+                                    const uint32_t pk[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+                                    float kf[16];
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) {
+                                        kf[2 * e] = __uint_as_float(pk[e] << 16);
+                                        kf[2 * e + 1] = __uint_as_float(pk[e] & 0xffff0000u);
+                                    }
+                                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                                    for (int e = 0; e < 16; e += 4) {
+                                        s0 = fmaf(kf[e], w[e], s0); s1 = fmaf(kf[e + 1], w[e + 1], s1);
+                                        s2 = fmaf(kf[e + 2], w[e + 2], s2); s3 = fmaf(kf[e + 3], w[e + 3], s3);
+                                    }
+                                    float sr = (s0 + s1) + (s2 + s3);
+                                    sr += __shfl_xor_sync(0xffffffffu, sr, 1);
+                                    sr += __shfl_xor_sync(0xffffffffu, sr, 2);
+                                    const float u = t * kTileRows + rin < g.nvalid ? __fdividef(1.f, sr) : 0.f;
+#pragma unroll
+                                    for (int e = 0; e < 16; ++e) c[e] = fmaf(kf[e], u, c[e]);
+                                }
+                            }
+                            // all four warps have the tile in registers: hand the stage back to the producer
+                            named_bar_sync(1 + grp, 128);
+                            if (gtid == 0 && ok) mbar_arrive(bar(bXEmpty + stg));
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) c[j] *= w[j];
+#pragma unroll
+                        for (int off = 4; off <= 16; off <<= 1) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) c[j] += __shfl_xor_sync(0xffffffffu, c[j], off);
+                        }
+                        if (ok) ok = wwait(bar(bSegEmpty + par), par_empty);
+                        if (rq == 0) {
+#pragma unroll
+                            for (int j = 0; j < 16; j += 2)
+                                *reinterpret_cast<float4 *>(dstp + (cq * 16 + j) * 2) = make_float4(0.f, c[j], 0.f, c[j + 1]);
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(bSegFull + par));
+                        continue;
+                    }
+                }
+                // first pass of a solve that will run stored-kernel passes: keep 2^(L - rowmax) as bf16
+                const bool store_kt = RP == 64 && P.Kt != nullptr && g.attempt == 0 && li < kMaxLoc;
 
                 auto run = [&](auto rbtag) {
                     constexpr bool RB = decltype(rbtag)::value;
@@ -760,7 +880,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         acc[ci] = 0.f;
                         if (RB) kap[ci] = neg_inf();
                     }
-                    for (int t = g.t0; t < g.t1; ++t, ++k) {
+                    for (int t = g.t0; t < g.t1; ++t, ++k, ++kx) {
                         const bool mine = gk == grp;
                         gk = gk + 1 == kGroups ? 0 : gk + 1;
                         if (!mine) continue;
@@ -807,6 +927,15 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                                     sB0 += ex2(v[rep * 4 + 2] - mB); sB1 += ex2(v[rep * 4 + 3] - mB);
                                 }
                             }
+                            if (!RB && store_kt) {
+                                // G = 0 in this pass, so the exponentials are the stored kernel's entries
+                                __nv_bfloat16 *kt = P.Kt + ((size_t)idx * P.npad + (size_t)t * kTileRows + qd * 32 + half * 16 + rq) * 64 + 2 * cq;
+#pragma unroll
+                                for (int rep = 0; rep < NC / 2; ++rep) {
+                                    *reinterpret_cast<uint32_t *>(kt + rep * 8) = pack_bf16(v[rep * 4 + 0], v[rep * 4 + 1]);
+                                    *reinterpret_cast<uint32_t *>(kt + 8 * 64 + rep * 8) = pack_bf16(v[rep * 4 + 2], v[rep * 4 + 3]);
+                                }
+                            }
                             float sA = sA0 + sA1, sB = sB0 + sB1;
                             sA += __shfl_xor_sync(0xffffffffu, sA, 1);
                             sB += __shfl_xor_sync(0xffffffffu, sB, 1);
@@ -848,6 +977,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             }
                         }
                     }
+                    if (store_kt) asm volatile("fence.proxy.async.global;" ::: "memory");
                     if (ok) ok = wwait(bar(bSegEmpty + par), par_empty);
                     if (rq == 0) {
 #pragma unroll
@@ -904,6 +1034,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             for (int t = g.t0; t < g.t1; ++t, ++k) {
                 const int pb = ka & 1, pj = ka >> 1, ob = ko & 1, oj = ko >> 1;
                 ++ka;
+                kx += WRED ? 2 : 1;
                 if (!WRED) ++ko;
                 const bool mine = gk == grp;
                 gk = gk + 1 == kGroups ? 0 : gk + 1;
@@ -1205,6 +1336,7 @@ FusedLayout fused_layout(int B, int H, int n, int d, int r)
     L.Wb = o; o += up256((size_t)BH * 2 * d * 64 * 2);
     L.part = o; o += up256((size_t)2 * 2 * BH * ms * RP * 2 * 8);
     L.head_end = o;
+    L.kt = o; o += RP == 64 ? up256((size_t)2 * BH * ((n + 127) / 128) * 128 * 64 * 2) : 0;
     L.zprep = o; o += up256((size_t)H * 2 * RP * d * 2);
     L.wpart = o; o += up256((size_t)BH * ms * 128 * d * 4);
     L.total = o;
@@ -1244,6 +1376,9 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
     if (!make_map(&P.tmQ, q, BH, n, d, 128) || !make_map(&P.tmK, k, BH, n, d, 128) ||
         !make_map(&P.tmV, v, BH, n, d, 128) || !make_map(&P.tmZ, zp, 2 * H, RP, d, RP))
         return cudaErrorInvalidValue;
+    P.npad = ((n + 127) / 128) * 128;
+    P.Kt = (RP == 64 && iters > 1) ? reinterpret_cast<__nv_bfloat16 *>(w + L.kt) : nullptr;
+    if (P.Kt != nullptr && !make_map(&P.tmKt, P.Kt, 2 * BH, P.npad, 64, 128)) return cudaErrorInvalidValue;
     P.beta = beta; P.key_len = key_len;
     P.G = reinterpret_cast<float *>(w + L.G);
     P.part = reinterpret_cast<unsigned long long *>(w + L.part);

@@ -89,8 +89,11 @@ def _check_full(x, want_g=True):
     err = worst_head_err(res["out"], ref)
     assert err <= TOL[x.q.dtype], f"{x.name} {x.q.dtype}: {err}"
     if want_g:
+        # potentials: float32 tensors 1e-4; bf16 tensors 1e-3, because passes 2..T of the fused bf16 path read the
+        # Gibbs kernel exp(C/eps - rowmax) back as bf16 (relative rounding 2^-9 per entry, averaged over the tokens)
+        gtol = 1e-4 if x.q.dtype == torch.float32 else 1e-3
         sc = max(1.0, np.abs(g1).max(), np.abs(g2).max())
-        assert np.abs(res["g1"] - g1).max() <= 1e-4 * sc and np.abs(res["g2"] - g2).max() <= 1e-4 * sc
+        assert np.abs(res["g1"] - g1).max() <= gtol * sc and np.abs(res["g2"] - g2).max() <= gtol * sc
     return err
 
 
