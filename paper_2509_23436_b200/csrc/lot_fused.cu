@@ -810,13 +810,11 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
 #pragma unroll
                         for (int j = 0; j < 16; ++j) w[j] = ex2(w[j] - gmax);
-                        int lt = 0;
-                        for (int t = g.t0; t < g.t1; ++t, ++k, ++kx) {
-                            const bool mine = lt == grp;
-                            lt = lt + 1 == kGroups ? 0 : lt + 1;
-                            if (!mine) continue;
-                            const int stg = kx % kStages;
-                            if (ok) ok = wwait(bar(bXFull + stg), (kx / kStages) & 1);
+                        // tile t0 + j goes to group j % kGroups: step straight from own tile to own tile
+                        for (int t = g.t0 + grp; t < g.t1; t += kGroups) {
+                            const int kxt = kx + (t - g.t0);
+                            const int stg = kxt % kStages;
+                            if (ok) ok = wwait(bar(bXFull + stg), (kxt / kStages) & 1);
                             if (ok) {
                                 const uint8_t *tile = smem + PL::offX + stg * kStageBytes;
 #pragma unroll
@@ -849,6 +847,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             named_bar_sync(1 + grp, 128);
                             if (gtid == 0 && ok) mbar_arrive(bar(bXEmpty + stg));
                         }
+                        k += g.t1 - g.t0;
+                        kx += g.t1 - g.t0;
 #pragma unroll
                         for (int j = 0; j < 16; ++j) c[j] *= w[j];
 #pragma unroll
@@ -880,10 +880,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         acc[ci] = 0.f;
                         if (RB) kap[ci] = neg_inf();
                     }
-                    for (int t = g.t0; t < g.t1; ++t, ++k, ++kx) {
-                        const bool mine = gk == grp;
-                        gk = gk + 1 == kGroups ? 0 : gk + 1;
-                        if (!mine) continue;
+                    // tile k goes to group k % kGroups: step straight from own tile to own tile
+                    const int first = grp >= gk ? grp - gk : grp - gk + kGroups;
+                    for (int t = g.t0 + first; t < g.t1; t += kGroups) {
                         if (ok) ok = wwait(bar(bAccFull + grp), mypar);
                         mypar ^= 1u;
                         if (!ok) continue;
@@ -963,6 +962,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             }
                         }
                     }
+                    gk = (gk + (g.t1 - g.t0)) % kGroups;
+                    k += g.t1 - g.t0;
+                    kx += g.t1 - g.t0;
                     // ---- warp partial: the 8 rows-lanes of every column quarter, left in shared memory
 #pragma unroll
                     for (int off = 4; off <= 16; off <<= 1) {
@@ -1031,14 +1033,10 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             // the tile loop is compiled once per pass kind, so that the other kind's work is not carried along
             auto tiles = [&](auto wtag) {
                 constexpr bool WRED = decltype(wtag)::value;
-            for (int t = g.t0; t < g.t1; ++t, ++k) {
-                const int pb = ka & 1, pj = ka >> 1, ob = ko & 1, oj = ko >> 1;
-                ++ka;
-                kx += WRED ? 2 : 1;
-                if (!WRED) ++ko;
-                const bool mine = gk == grp;
-                gk = gk + 1 == kGroups ? 0 : gk + 1;
-                if (!mine) continue;
+            const int first = grp >= gk ? grp - gk : grp - gk + kGroups;
+            for (int t = g.t0 + first; t < g.t1; t += kGroups) {
+                const int kat = ka + (t - g.t0), kot = ko + (t - g.t0);
+                const int pb = kat & 1, pj = kat >> 1, ob = kot & 1, oj = kot >> 1;
                 if (ok) ok = wwait(bar(bAccFull + grp), mypar);
                 mypar ^= 1u;
                 if (!ok) continue;
@@ -1124,6 +1122,12 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     }
                 }
             }
+            {
+                const int nt = g.t1 - g.t0;
+                gk = (gk + nt) % kGroups;
+                k += nt; ka += nt; kx += WRED ? 2 * nt : nt;
+                if (!WRED) ko += nt;
+            }
             };
             if (g.phase == kPhaseWred) tiles(std::true_type{});
             else tiles(std::false_type{});
@@ -1167,10 +1171,10 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         const float bt = tt < P.r ? __ldg(P.beta + g.h * P.r + tt) : 1.f;   // issued with the partial loads
                         float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
                         const float *src0 = P.wpart + ((size_t)g.s * P.maxslots * 128) * DK + c;
-                        for (int sl0 = 0; sl0 < g.nslots; sl0 += 12) {
-                            float4 a[12], b[12];
+                        for (int sl0 = 0; sl0 < g.nslots; sl0 += 6) {
+                            float4 a[6], b[6];
 #pragma unroll
-                            for (int u = 0; u < 12; ++u) {
+                            for (int u = 0; u < 6; ++u) {
                                 a[u] = b[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                                 if (sl0 + u < g.nslots) {
                                     const float *src = src0 + ((size_t)(sl0 + u) * 128) * DK;
@@ -1179,7 +1183,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                                 }
                             }
 #pragma unroll
-                            for (int u = 0; u < 12; ++u) {
+                            for (int u = 0; u < 6; ++u) {
                                 sum.x += a[u].x + b[u].x; sum.y += a[u].y + b[u].y;
                                 sum.z += a[u].z + b[u].z; sum.w += a[u].w + b[u].w;
                             }
