@@ -797,19 +797,21 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         // w_t = 2^(G_t - max G) the row sums are s_i = sum_t K~_it w_t and the column sums
                         // w_t sum_i K~_it / s_i: two FMAs per entry, no exponential, no tensor-core work.
                         // Thread = 4 rows (rq + 8 j of the warp's 32) x 16 consecutive columns (16 cq ..).
-                        float w[16], c[16];
+                        // column pairs are kept as float2 so that the sums run as packed two-wide FMAs
+                        float2 w2[8], c2[8];
                         float gmax = neg_inf();
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int col = cq * 16 + j;
-                            w[j] = col < P.r ? sGc[li * 64 + col] : neg_inf();
-                            gmax = fmaxf(gmax, w[j]);
-                            c[j] = 0.f;
+                        for (int j = 0; j < 8; ++j) {
+                            const int col = cq * 16 + 2 * j;
+                            w2[j].x = col < P.r ? sGc[li * 64 + col] : neg_inf();
+                            w2[j].y = col + 1 < P.r ? sGc[li * 64 + col + 1] : neg_inf();
+                            gmax = max3(gmax, w2[j].x, w2[j].y);
+                            c2[j] = make_float2(0.f, 0.f);
                         }
                         gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
                         gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) w[j] = ex2(w[j] - gmax);
+                        for (int j = 0; j < 8; ++j) { w2[j].x = ex2(w2[j].x - gmax); w2[j].y = ex2(w2[j].y - gmax); }
                         // tile t0 + j goes to group j % kGroups: step straight from own tile to own tile
                         for (int t = g.t0 + grp; t < g.t1; t += kGroups) {
                             const int kxt = kx + (t - g.t0);
@@ -823,24 +825,23 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                                     const uint4 a = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq) ^ (rin & 7)) * 16));
                                     const uint4 b = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq + 1) ^ (rin & 7)) * 16));
                                     const uint32_t pk[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-                                    float kf[16];
+                                    float2 kf[8];
 #pragma unroll
-                                    for (int e = 0; e < 8; ++e) {
-                                        kf[2 * e] = __uint_as_float(pk[e] << 16);
-                                        kf[2 * e + 1] = __uint_as_float(pk[e] & 0xffff0000u);
-                                    }
-                                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                                    for (int e = 0; e < 8; ++e)
+                                        kf[e] = make_float2(__uint_as_float(pk[e] << 16), __uint_as_float(pk[e] & 0xffff0000u));
+                                    float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
 #pragma unroll
-                                    for (int e = 0; e < 16; e += 4) {
-                                        s0 = fmaf(kf[e], w[e], s0); s1 = fmaf(kf[e + 1], w[e + 1], s1);
-                                        s2 = fmaf(kf[e + 2], w[e + 2], s2); s3 = fmaf(kf[e + 3], w[e + 3], s3);
+                                    for (int e = 0; e < 8; e += 2) {
+                                        sa = __ffma2_rn(kf[e], w2[e], sa);
+                                        sb = __ffma2_rn(kf[e + 1], w2[e + 1], sb);
                                     }
-                                    float sr = (s0 + s1) + (s2 + s3);
+                                    float sr = (sa.x + sa.y) + (sb.x + sb.y);
                                     sr += __shfl_xor_sync(0xffffffffu, sr, 1);
                                     sr += __shfl_xor_sync(0xffffffffu, sr, 2);
                                     const float u = t * kTileRows + rin < g.nvalid ? __fdividef(1.f, sr) : 0.f;
+                                    const float2 uu = make_float2(u, u);
 #pragma unroll
-                                    for (int e = 0; e < 16; ++e) c[e] = fmaf(kf[e], u, c[e]);
+                                    for (int e = 0; e < 8; ++e) c2[e] = __ffma2_rn(kf[e], uu, c2[e]);
                                 }
                             }
                             // all four warps have the tile in registers: hand the stage back to the producer
@@ -849,8 +850,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         }
                         k += g.t1 - g.t0;
                         kx += g.t1 - g.t0;
+                        float c[16];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) c[j] *= w[j];
+                        for (int j = 0; j < 8; ++j) { c[2 * j] = c2[j].x * w2[j].x; c[2 * j + 1] = c2[j].y * w2[j].y; }
 #pragma unroll
                         for (int off = 4; off <= 16; off <<= 1) {
 #pragma unroll
