@@ -274,6 +274,40 @@ __device__ __forceinline__ void ld_tagged(const unsigned long long *p, unsigned 
     asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(p) : "memory");
 }
 
+// Sum a[0..15] over the 8 lanes that share (lane & 3), halving the live set in every round (14 shuffles instead of
+// 48).  Afterwards every lane holds in a[0], a[1] the totals of entries b, b + 1; b is returned.
+template <int N>
+__device__ __forceinline__ int quad_col_reduce16(float (&a)[N], int lane)
+{
+    if constexpr (N == 16) {
+    {
+        const bool up = (lane & 16) != 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float send = up ? a[j] : a[j + 8], keep = up ? a[j + 8] : a[j];
+            a[j] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+        }
+    }
+    {
+        const bool up = (lane & 8) != 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float send = up ? a[j] : a[j + 4], keep = up ? a[j + 4] : a[j];
+            a[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+    }
+    {
+        const bool up = (lane & 4) != 0;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const float send = up ? a[j] : a[j + 2], keep = up ? a[j + 2] : a[j];
+            a[j] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+        }
+    }
+    }
+    return 8 * ((lane >> 4) & 1) + 4 * ((lane >> 3) & 1) + 2 * ((lane >> 2) & 1);
+}
+
 // Quad-layout TMEM load (16 lanes x RP columns): thread L of the warp gets, in v[rep*4 + k],
 // lane L/4 + 8*(k/2) and column rep*8 + 2*(L%4) + (k%2) of the 16-lane block at taddr.
 template <int RP>
@@ -801,12 +835,17 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         float2 w2[8], c2[8];
                         float gmax = neg_inf();
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
+                        for (int j = 0; j < 8; j += 2) {
                             const int col = cq * 16 + 2 * j;
-                            w2[j].x = col < P.r ? sGc[li * 64 + col] : neg_inf();
-                            w2[j].y = col + 1 < P.r ? sGc[li * 64 + col + 1] : neg_inf();
+                            const float4 g4 = *reinterpret_cast<const float4 *>(sGc + li * 64 + col);
+                            w2[j].x = col < P.r ? g4.x : neg_inf();
+                            w2[j].y = col + 1 < P.r ? g4.y : neg_inf();
+                            w2[j + 1].x = col + 2 < P.r ? g4.z : neg_inf();
+                            w2[j + 1].y = col + 3 < P.r ? g4.w : neg_inf();
                             gmax = max3(gmax, w2[j].x, w2[j].y);
+                            gmax = max3(gmax, w2[j + 1].x, w2[j + 1].y);
                             c2[j] = make_float2(0.f, 0.f);
+                            c2[j + 1] = make_float2(0.f, 0.f);
                         }
                         gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
                         gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
@@ -853,17 +892,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         float c[16];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) { c[2 * j] = c2[j].x * w2[j].x; c[2 * j + 1] = c2[j].y * w2[j].y; }
-#pragma unroll
-                        for (int off = 4; off <= 16; off <<= 1) {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) c[j] += __shfl_xor_sync(0xffffffffu, c[j], off);
-                        }
+                        const int cb = quad_col_reduce16(c, lane);
                         if (ok) ok = wwait(bar(bSegEmpty + par), par_empty);
-                        if (rq == 0) {
-#pragma unroll
-                            for (int j = 0; j < 16; j += 2)
-                                *reinterpret_cast<float4 *>(dstp + (cq * 16 + j) * 2) = make_float4(0.f, c[j], 0.f, c[j + 1]);
-                        }
+                        *reinterpret_cast<float4 *>(dstp + (cq * 16 + cb) * 2) = make_float4(0.f, c[0], 0.f, c[1]);
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar(bSegFull + par));
                         continue;
@@ -968,6 +999,15 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     k += g.t1 - g.t0;
                     kx += g.t1 - g.t0;
                     // ---- warp partial: the 8 rows-lanes of every column quarter, left in shared memory
+                    if constexpr (!RB && NC == 16) {
+                        const int cb = quad_col_reduce16(acc, lane);
+                        if (store_kt) asm volatile("fence.proxy.async.global;" ::: "memory");
+                        if (ok) ok = wwait(bar(bSegEmpty + par), par_empty);
+                        *reinterpret_cast<float4 *>(dstp + ((cb >> 1) * 8 + 2 * cq) * 2) = make_float4(0.f, acc[0], 0.f, acc[1]);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(bSegFull + par));
+                        return;
+                    }
 #pragma unroll
                     for (int off = 4; off <= 16; off <<= 1) {
 #pragma unroll
