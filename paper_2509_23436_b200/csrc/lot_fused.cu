@@ -506,7 +506,10 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         uint32_t gpar = 0;
         int ka = 0, ko = 0;                   // tiles of the apply passes / of the OUT pass so far
         bool ok = true, w_open = false;
-        int pend_k = -1, pend_o = 0, pend_first = 0, pend_vs = 0, pend_phase = 0;   // apply MMA still to be issued
+        // Apply MMAs are issued two tiles late, so that three tiles (one per epilogue group) are in flight:
+        // pend_* is the older waiting tile, pnew_* the newer one.
+        int pend_k = -1, pend_o = 0, pend_first = 0, pend_vs = 0, pend_phase = 0;
+        int pnew_k = -1, pnew_o = 0, pnew_first = 0, pnew_vs = 0, pnew_phase = 0;
         const uint32_t tm = __shfl_sync(0xffffffffu, tmem_base, 0);
         // Descriptors differ only in the 16-byte-granular start address (low word).
         const uint64_t dK = make_smem_desc(sbase, 16, 1024);               // K-major operand, 128-byte rows
@@ -548,7 +551,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 }
             }
             __syncwarp();
-            pend_k = -1;
+            pend_k = pnew_k; pend_o = pnew_o; pend_first = pnew_first; pend_vs = pnew_vs; pend_phase = pnew_phase;
+            pnew_k = -1;
         };
 
         while (ok && it.next(g)) {
@@ -565,7 +569,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     continue;
                 }
             }
-            if (pend_k >= 0) issue_apply();
+            while (pend_k >= 0) issue_apply();
             if (w_open) {                                                    // W of the previous WRED segment complete
                 if (ok && elect_one()) umma_commit(bar(bWFull));
                 __syncwarp();
@@ -616,13 +620,14 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 if (g.phase != kPhaseSum) {
                     const int vs = kx;
                     if (g.phase == kPhaseWred) ++kx;      // the value tile sits in the next ring stage
-                    if (pend_k >= 0) issue_apply();
-                    pend_k = ka++; pend_first = (t == g.t0); pend_vs = vs; pend_phase = g.phase;
-                    if (g.phase == kPhaseOut) pend_o = ko++;
+                    if (pnew_k >= 0) issue_apply();          // two waiting already: issue the older one
+                    const int nk = ka++, no = g.phase == kPhaseOut ? ko++ : 0;
+                    if (pend_k < 0) { pend_k = nk; pend_o = no; pend_first = (t == g.t0); pend_vs = vs; pend_phase = g.phase; }
+                    else { pnew_k = nk; pnew_o = no; pnew_first = (t == g.t0); pnew_vs = vs; pnew_phase = g.phase; }
                 }
             }
         }
-        if (pend_k >= 0 && ok) issue_apply();
+        while (pend_k >= 0 && ok) issue_apply();
         if (w_open && ok && elect_one()) umma_commit(bar(bWFull));
         __syncwarp();
     } else if (warp == 2) {
