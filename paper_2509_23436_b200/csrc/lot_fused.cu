@@ -202,7 +202,8 @@ struct Plan {
 
 enum BarId { bXFull = 0, bXEmpty = 8, bZFull = 16, bZEmpty = 18, bAccFull = 20, bAccEmpty = 24, bPFull = 28, bPEmpty = 30,
              bOFull = 32, bOEmpty = 34, bWFull = 36, bWEmpty = 37, bWqFull = 38, bWqEmpty = 39, bSegFull = 40, bSegEmpty = 42,
-             bCount = 44 };
+             bREmpty = 44,   // stage released by the four warps that read a stored-kernel tile (bXEmpty: by an MMA commit)
+             bCount = 52 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 {
@@ -380,7 +381,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     const int BH = P.B * P.H;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(bar(bXFull + i), 1); mbar_init(bar(bXEmpty + i), 1); }
+        for (int i = 0; i < kStages; ++i) { mbar_init(bar(bXFull + i), 1); mbar_init(bar(bXEmpty + i), 1); mbar_init(bar(bREmpty + i), 4); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(bZFull + i), 1); mbar_init(bar(bZEmpty + i), 1);
             mbar_init(bar(bPFull + i), 4); mbar_init(bar(bPEmpty + i), 1);
@@ -432,6 +433,21 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             Seg g;
             int kx = 0, ztag[2] = {-1, -1}, zuse[2] = {0, 0};
             bool ok = true;
+            // A stage is handed back either by an MMA commit (bXEmpty) or by the readers of a stored-kernel tile
+            // (bREmpty): remember per stage which one its last use ends with and how often each has happened.
+            uint32_t used = 0, lastres = 0, xpar = 0, rpar = 0;     // bit st: used at all / last use was a kernel tile /
+                                                                    // parity of the commit-released / reader-released uses
+            auto acquire_stage = [&](int st, bool res) -> bool {
+                bool w = true;
+                if (used & (1u << st)) {
+                    if (lastres & (1u << st)) w = mbar_wait(bar(bREmpty + st), ((rpar >> st) & 1) ^ 1, sAbort, P.status);
+                    else w = mbar_wait(bar(bXEmpty + st), ((xpar >> st) & 1) ^ 1, sAbort, P.status);
+                }
+                used |= 1u << st;
+                if (res) { lastres |= 1u << st; rpar ^= 1u << st; }
+                else { lastres &= ~(1u << st); xpar ^= 1u << st; }
+                return w;
+            };
             while (ok && it.next(g)) {
                 const int idx = g.side * BH + g.s;
                 bool resident = false;
@@ -444,8 +460,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 if (resident) {
                     // tiles of the stored Gibbs kernel instead of token tiles; no pivots, no MMA
                     for (int t = g.t0; t < g.t1 && ok; ++t) {
-                        const int st = kx % kStages, ph = (kx / kStages) & 1;
-                        ok = mbar_wait(bar(bXEmpty + st), ph ^ 1, sAbort, P.status);
+                        const int st = kx % kStages;
+                        ok = acquire_stage(st, true);
                         if (!ok) break;
                         mbar_arrive_expect_tx(bar(bXFull + st), kStageBytes);
                         tma_load_3d(sbase + PL::offX + st * kStageBytes, &P.tmKt, bar(bXFull + st), 0, t * kTileRows, idx);
@@ -467,16 +483,16 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 const CUtensorMap *xm = g.side ? &P.tmK : &P.tmQ;
                 for (int t = g.t0; t < g.t1 && ok; ++t) {
                     {
-                        const int st = kx % kStages, ph = (kx / kStages) & 1;
-                        ok = mbar_wait(bar(bXEmpty + st), ph ^ 1, sAbort, P.status);
+                        const int st = kx % kStages;
+                        ok = acquire_stage(st, false);
                         if (!ok) break;
                         mbar_arrive_expect_tx(bar(bXFull + st), kStageBytes);
                         tma_load_3d(sbase + PL::offX + st * kStageBytes, xm, bar(bXFull + st), 0, t * kTileRows, g.s);
                         ++kx;
                     }
                     if (g.phase == kPhaseWred) {
-                        const int st = kx % kStages, ph = (kx / kStages) & 1;
-                        ok = mbar_wait(bar(bXEmpty + st), ph ^ 1, sAbort, P.status);
+                        const int st = kx % kStages;
+                        ok = acquire_stage(st, false);
                         if (!ok) break;
                         mbar_arrive_expect_tx(bar(bXFull + st), kStageBytes);
                         tma_load_3d(sbase + PL::offX + st * kStageBytes, &P.tmV, bar(bXFull + st), 0, t * kTileRows, g.s);
@@ -888,9 +904,9 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                                     for (int e = 0; e < 8; ++e) c2[e] = __ffma2_rn(kf[e], uu, c2[e]);
                                 }
                             }
-                            // all four warps have the tile in registers: hand the stage back to the producer
-                            named_bar_sync(1 + grp, 128);
-                            if (gtid == 0 && ok) mbar_arrive(bar(bXEmpty + stg));
+                            // this warp has its rows in registers: one of the four releases of the stage
+                            __syncwarp();
+                            if (lane == 0 && ok) mbar_arrive(bar(bREmpty + stg));
                         }
                         k += g.t1 - g.t0;
                         kx += g.t1 - g.t0;
