@@ -880,28 +880,47 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             if (ok) {
                                 const uint8_t *tile = smem + PL::offX + stg * kStageBytes;
 #pragma unroll
-                                for (int jr = 0; jr < 4; ++jr) {
-                                    const int rin = w4 * 32 + jr * 8 + rq;           // row inside the tile
-                                    const uint4 a = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq) ^ (rin & 7)) * 16));
-                                    const uint4 b = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq + 1) ^ (rin & 7)) * 16));
-                                    const uint32_t pk[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-                                    float2 kf[8];
+                                for (int jp = 0; jp < 4; jp += 2) {
+                                    // two rows advance in step: every instruction has an independent twin
+                                    float2 kf[2][8], sa[2], sb[2];
+                                    float sr[2];
 #pragma unroll
-                                    for (int e = 0; e < 8; ++e)
-                                        kf[e] = make_float2(__uint_as_float(pk[e] << 16), __uint_as_float(pk[e] & 0xffff0000u));
-                                    float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
+                                    for (int q = 0; q < 2; ++q) {
+                                        const int rin = w4 * 32 + (jp + q) * 8 + rq;           // row inside the tile
+                                        const uint4 a = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq) ^ (rin & 7)) * 16));
+                                        const uint4 b = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq + 1) ^ (rin & 7)) * 16));
+                                        const uint32_t pk[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+                                        for (int e = 0; e < 8; ++e)
+                                            kf[q][e] = make_float2(__uint_as_float(pk[e] << 16), __uint_as_float(pk[e] & 0xffff0000u));
+                                        sa[q] = make_float2(0.f, 0.f); sb[q] = make_float2(0.f, 0.f);
+                                    }
 #pragma unroll
                                     for (int e = 0; e < 8; e += 2) {
-                                        sa = __ffma2_rn(kf[e], w2[e], sa);
-                                        sb = __ffma2_rn(kf[e + 1], w2[e + 1], sb);
-                                    }
-                                    float sr = (sa.x + sa.y) + (sb.x + sb.y);
-                                    sr += __shfl_xor_sync(0xffffffffu, sr, 1);
-                                    sr += __shfl_xor_sync(0xffffffffu, sr, 2);
-                                    const float u = t * kTileRows + rin < g.nvalid ? __fdividef(1.f, sr) : 0.f;
-                                    const float2 uu = make_float2(u, u);
 #pragma unroll
-                                    for (int e = 0; e < 8; ++e) c2[e] = __ffma2_rn(kf[e], uu, c2[e]);
+                                        for (int q = 0; q < 2; ++q) {
+                                            sa[q] = __ffma2_rn(kf[q][e], w2[e], sa[q]);
+                                            sb[q] = __ffma2_rn(kf[q][e + 1], w2[e + 1], sb[q]);
+                                        }
+                                    }
+#pragma unroll
+                                    for (int q = 0; q < 2; ++q) sr[q] = (sa[q].x + sa[q].y) + (sb[q].x + sb[q].y);
+#pragma unroll
+                                    for (int q = 0; q < 2; ++q) sr[q] += __shfl_xor_sync(0xffffffffu, sr[q], 1);
+#pragma unroll
+                                    for (int q = 0; q < 2; ++q) sr[q] += __shfl_xor_sync(0xffffffffu, sr[q], 2);
+                                    float2 uu[2];
+#pragma unroll
+                                    for (int q = 0; q < 2; ++q) {
+                                        const int rin = w4 * 32 + (jp + q) * 8 + rq;
+                                        const float u = t * kTileRows + rin < g.nvalid ? __fdividef(1.f, sr[q]) : 0.f;
+                                        uu[q] = make_float2(u, u);
+                                    }
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) {
+                                        c2[e] = __ffma2_rn(kf[0][e], uu[0], c2[e]);
+                                        c2[e] = __ffma2_rn(kf[1][e], uu[1], c2[e]);
+                                    }
                                 }
                             }
                             // this warp has its rows in registers: one of the four releases of the stage
