@@ -140,7 +140,7 @@ struct Sched {
     const FusedParams &P;
     const int *tab;
     int u0, u1, s_lo, s_hi, nloc, pass, cur;
-    __device__ Sched(const FusedParams &p, const int *table) : P(p), tab(table)
+    __device__ __forceinline__ Sched(const FusedParams &p, const int *table) : P(p), tab(table)
     {
         cta_range(p, blockIdx.x, u0, u1);
         s_lo = u0 / p.TPS;
@@ -150,7 +150,7 @@ struct Sched {
         pass = p.T == 0 ? 1 : 0;       // passes 0..T-1 SUM, T spare SUM, T+1 WRED, T+2 OUT
         cur = 0;
     }
-    __device__ bool next(Seg &g)
+    __device__ __forceinline__ bool next(Seg &g)
     {
         for (;;) {
             if (pass > P.T + 2) return false;
@@ -974,10 +974,12 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             float mA = neg_inf(), mB = neg_inf();
 #pragma unroll
                             for (int rep = 0; rep < NC / 2; ++rep) {
-                                v[rep * 4 + 0] += Gr[rep * 2]; v[rep * 4 + 1] += Gr[rep * 2 + 1];
-                                v[rep * 4 + 2] += Gr[rep * 2]; v[rep * 4 + 3] += Gr[rep * 2 + 1];
-                                mA = max3(mA, v[rep * 4 + 0], v[rep * 4 + 1]);
-                                mB = max3(mB, v[rep * 4 + 2], v[rep * 4 + 3]);
+                                const float2 g2 = make_float2(Gr[rep * 2], Gr[rep * 2 + 1]);
+                                const float2 xa = __fadd2_rn(make_float2(v[rep * 4 + 0], v[rep * 4 + 1]), g2);
+                                const float2 xb = __fadd2_rn(make_float2(v[rep * 4 + 2], v[rep * 4 + 3]), g2);
+                                v[rep * 4 + 0] = xa.x; v[rep * 4 + 1] = xa.y; v[rep * 4 + 2] = xb.x; v[rep * 4 + 3] = xb.y;
+                                mA = max3(mA, xa.x, xa.y);
+                                mB = max3(mB, xb.x, xb.y);
                             }
                             mA = fmaxf(mA, __shfl_xor_sync(0xffffffffu, mA, 1));
                             mB = fmaxf(mB, __shfl_xor_sync(0xffffffffu, mB, 1));
@@ -985,13 +987,19 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             mB = fmaxf(mB, __shfl_xor_sync(0xffffffffu, mB, 2));
                             float sA0 = 0.f, sA1 = 0.f, sB0 = 0.f, sB1 = 0.f;
                             if (!RB) {
+                                // column pairs as packed two-wide operations
+                                const float2 nA = make_float2(-mA, -mA), nB = make_float2(-mB, -mB);
+                                float2 sA2 = make_float2(0.f, 0.f), sB2 = make_float2(0.f, 0.f);
 #pragma unroll
                                 for (int rep = 0; rep < NC / 2; ++rep) {
-                                    v[rep * 4 + 0] = ex2(v[rep * 4 + 0] - mA); sA0 += v[rep * 4 + 0];
-                                    v[rep * 4 + 1] = ex2(v[rep * 4 + 1] - mA); sA1 += v[rep * 4 + 1];
-                                    v[rep * 4 + 2] = ex2(v[rep * 4 + 2] - mB); sB0 += v[rep * 4 + 2];
-                                    v[rep * 4 + 3] = ex2(v[rep * 4 + 3] - mB); sB1 += v[rep * 4 + 3];
+                                    const float2 xa = __fadd2_rn(make_float2(v[rep * 4 + 0], v[rep * 4 + 1]), nA);
+                                    const float2 xb = __fadd2_rn(make_float2(v[rep * 4 + 2], v[rep * 4 + 3]), nB);
+                                    const float2 ea = make_float2(ex2(xa.x), ex2(xa.y)), eb = make_float2(ex2(xb.x), ex2(xb.y));
+                                    v[rep * 4 + 0] = ea.x; v[rep * 4 + 1] = ea.y; v[rep * 4 + 2] = eb.x; v[rep * 4 + 3] = eb.y;
+                                    sA2 = __fadd2_rn(sA2, ea);
+                                    sB2 = __fadd2_rn(sB2, eb);
                                 }
+                                sA0 = sA2.x; sA1 = sA2.y; sB0 = sB2.x; sB1 = sB2.y;
                             } else {
 #pragma unroll
                                 for (int rep = 0; rep < NC / 2; ++rep) {
@@ -1016,10 +1024,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             if (!RB) {
                                 const float wA = rowA < g.nvalid ? __fdividef(1.f, sA) : 0.f;
                                 const float wB = rowB < g.nvalid ? __fdividef(1.f, sB) : 0.f;
+                                const float2 wA2 = make_float2(wA, wA), wB2 = make_float2(wB, wB);
 #pragma unroll
-                                for (int ci = 0; ci < NC; ++ci) {
-                                    acc[ci] = fmaf(v[(ci >> 1) * 4 + (ci & 1)], wA, acc[ci]);
-                                    acc[ci] = fmaf(v[(ci >> 1) * 4 + 2 + (ci & 1)], wB, acc[ci]);
+                                for (int rep = 0; rep < NC / 2; ++rep) {
+                                    float2 a2 = make_float2(acc[rep * 2], acc[rep * 2 + 1]);
+                                    a2 = __ffma2_rn(make_float2(v[rep * 4 + 0], v[rep * 4 + 1]), wA2, a2);
+                                    a2 = __ffma2_rn(make_float2(v[rep * 4 + 2], v[rep * 4 + 3]), wB2, a2);
+                                    acc[rep * 2] = a2.x; acc[rep * 2 + 1] = a2.y;
                                 }
                             } else {
                                 // exact log2 of every normalised entry, added to (kappa, S) pairs
