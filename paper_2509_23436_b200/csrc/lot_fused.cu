@@ -190,7 +190,8 @@ struct Plan {
     static constexpr int offGc = offG + kGroups * 64 * 4;      // float sGc[kMaxLoc][64]: this CTA's copy of the potentials
     static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust, sMode [kMaxLoc]
     static constexpr int offSeg = offState + 4 * kMaxLoc * 4;  // int sSeg[kMaxLoc][kSegInts]: static parts of the segments
-    static constexpr int total = offSeg + kMaxLoc * kSegInts * 4;
+    static constexpr int offWt = offSeg + kMaxLoc * kSegInts * 4; // float sWt[kMaxLoc][64]: weights 2^(G - max G) of the stored-kernel passes
+    static constexpr int total = offWt + kMaxLoc * 64 * 4;
     // float sPart[2][kEpiWarps][64][2], the per-warp column pairs of the SUM passes, lives in the first plan buffer
     // (free until the WRED pass; the epilogue waits for the publisher's last read before it writes a plan tile)
     static constexpr int offPart = offP;
@@ -377,6 +378,14 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         return __all_sync(0xffffffffu, r) != 0;
     };
 
+    // the same for two barriers whose first tries are in flight together
+    auto wwait2 = [&](uint32_t b0, uint32_t p0, uint32_t b1, uint32_t p1) {
+        const bool r0 = mbar_try_wait(b0, p0);
+        const bool r1 = mbar_try_wait(b1, p1);
+        if (__all_sync(0xffffffffu, r0 && r1)) return true;
+        return wwait(b0, p0) && wwait(b1, p1);
+    };
+
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BH = P.B * P.H;
 
@@ -536,11 +545,10 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
 
         auto issue_apply = [&]() {
             const int pb = pend_k & 1, pj = pend_k >> 1, ob = pend_o & 1, oj = pend_o >> 1;
-            if (ok) ok = wwait(bar(bPFull + pb), pj & 1);
             const uint32_t pa = (PL::offP + pb * PL::PBYTES) >> 4;
             if (pend_phase == kPhaseWred) {
                 const int vs = pend_vs % kStages, vph = (pend_vs / kStages) & 1;
-                if (ok) ok = wwait(bar(bXFull + vs), vph);
+                if (ok) ok = wwait2(bar(bPFull + pb), pj & 1, bar(bXFull + vs), vph);
                 tc_fence_after();
                 const uint32_t va = (PL::offX + vs * kStageBytes) >> 4;
                 if (ok && elect_one()) {
@@ -552,7 +560,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     umma_commit(bar(bXEmpty + vs));
                 }
             } else {
-                if (ok) ok = wwait(bar(bOEmpty + ob), (oj & 1) ^ 1);
+                if (ok) ok = wwait2(bar(bPFull + pb), pj & 1, bar(bOEmpty + ob), (oj & 1) ^ 1);
                 tc_fence_after();
                 if (ok && elect_one()) {
 #pragma unroll
@@ -616,8 +624,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 gpar ^= 1u << grp;
                 gk = gk + 1 == kGroups ? 0 : gk + 1;
                 const int st = kx % kStages, ph = (kx / kStages) & 1;
-                ok = wwait(bar(bXFull + st), ph);
-                if (ok) ok = wwait(bar(bAccEmpty + grp), gbit ^ 1);
+                ok = wwait2(bar(bXFull + st), ph, bar(bAccEmpty + grp), gbit ^ 1);
                 tc_fence_after();
                 const uint32_t xa = dK_lo + ((PL::offX + st * kStageBytes) >> 4);
                 const uint32_t dcol = tm + grp * RP;
@@ -790,6 +797,12 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 gmn = fminf(gmn, __shfl_xor_sync(0xffffffffu, gmn, off));
             }
             const int next_resident = RP == 64 && cached && !fail && !rb && P.Kt != nullptr && (gmx - gmn) <= 64.f;
+            if (next_resident && mine) {
+                // weights of the next attempt, w_t = 2^(G_t - max G), computed once here for all epilogue warps
+                float *sWt = reinterpret_cast<float *>(smem + PL::offWt) + li * 64;
+                sWt[c0] = c0 < P.r ? ex2(sGc[li * 64 + c0] - gmx) : 0.f;
+                sWt[c0 + 1] = c0 + 1 < P.r ? ex2(sGc[li * 64 + c0 + 1] - gmx) : 0.f;
+            }
             if (cached) {
                 __threadfence_block();
                 __syncwarp();
@@ -854,24 +867,17 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         // Thread = 4 rows (rq + 8 j of the warp's 32) x 16 consecutive columns (16 cq ..).
                         // column pairs are kept as float2 so that the sums run as packed two-wide FMAs
                         float2 w2[8], c2[8];
-                        float gmax = neg_inf();
+                        {
+                            const float4 *wt = reinterpret_cast<const float4 *>(smem + PL::offWt + (li * 64 + cq * 16) * 4);
 #pragma unroll
-                        for (int j = 0; j < 8; j += 2) {
-                            const int col = cq * 16 + 2 * j;
-                            const float4 g4 = *reinterpret_cast<const float4 *>(sGc + li * 64 + col);
-                            w2[j].x = col < P.r ? g4.x : neg_inf();
-                            w2[j].y = col + 1 < P.r ? g4.y : neg_inf();
-                            w2[j + 1].x = col + 2 < P.r ? g4.z : neg_inf();
-                            w2[j + 1].y = col + 3 < P.r ? g4.w : neg_inf();
-                            gmax = max3(gmax, w2[j].x, w2[j].y);
-                            gmax = max3(gmax, w2[j + 1].x, w2[j + 1].y);
-                            c2[j] = make_float2(0.f, 0.f);
-                            c2[j + 1] = make_float2(0.f, 0.f);
+                            for (int j = 0; j < 4; ++j) {
+                                const float4 w4v = wt[j];
+                                w2[2 * j] = make_float2(w4v.x, w4v.y);
+                                w2[2 * j + 1] = make_float2(w4v.z, w4v.w);
+                                c2[2 * j] = make_float2(0.f, 0.f);
+                                c2[2 * j + 1] = make_float2(0.f, 0.f);
+                            }
                         }
-                        gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
-                        gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) { w2[j].x = ex2(w2[j].x - gmax); w2[j].y = ex2(w2[j].y - gmax); }
                         // tile t0 + j goes to group j % kGroups: step straight from own tile to own tile
                         for (int t = g.t0 + grp; t < g.t1; t += kGroups) {
                             const int kxt = kx + (t - g.t0);
