@@ -69,10 +69,8 @@ struct alignas(64) FusedParams {
     int *epoch;                  // [2][BH] attempts finished (used for segments beyond the shared-memory cache)
     int *iter;                   // [2][BH] pivot updates done
     int *robust;                 // [2][BH] 1 = column sums carried as (kappa, S) pairs (sticky)
-    float *wpart;                // [BH][maxslots][128][64] per-slot W accumulators (rows 0-63 hi, 64-127 lo)
-    __nv_bfloat16 *Wb;           // [BH][2][64][64] W'^T split hi/lo, pivot-contiguous
-    unsigned *wticket;           // [BH]
-    int *wdone;                  // [BH] 1 = Wb of the slice is final
+    float *wpart;                // [BH][maxslots][64 channels][64 pivots] per-slot partial of W^T = (Gamma2 V)^T
+    int *wflag;                  // [BH][maxslots] 1 = that slot's partial is complete
     __nv_bfloat16 *out;          // [BH][n][64]
     float *g_nat;                // [2][BH][r] final potentials, natural-log units
     int *status;
@@ -355,7 +353,6 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + PL::offBar);
     volatile int *sAbort = reinterpret_cast<volatile int *>(smem + PL::offMisc);
     uint32_t *sTmem = reinterpret_cast<uint32_t *>(smem + PL::offMisc + 4);
-    volatile int *sLastW = reinterpret_cast<volatile int *>(smem + PL::offMisc + 8);
     float *sG = reinterpret_cast<float *>(smem + PL::offG);
     float *sPart = reinterpret_cast<float *>(smem + PL::offPart);
     float *sGc = reinterpret_cast<float *>(smem + PL::offGc);
@@ -1101,11 +1098,17 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             if (gtid == 0) {
                 bool w = spin_ge(sPubDone, 1, sAbort, P.status);          // plan buffers free of SUM partials
                 if (w) w = li < kMaxLoc ? spin_ge(sIter + li, P.T, sAbort, P.status) : poll_ge(P.iter + idx, P.T, sAbort, P.status);
-                if (g.phase == kPhaseOut) {
-                    int kv = P.n;
-                    if (P.key_len != nullptr) kv = min(max(__ldg(P.key_len + g.b), 0), P.n);
-                    if (w && kv > 0) w = poll_ge(P.wdone + g.s, 1, sAbort, P.status);
+            }
+            // key-side geometry of this slice: which slots hold a partial of W
+            int kv = P.n, wslots = 0;
+            if (g.phase == kPhaseOut) {
+                if (P.key_len != nullptr) kv = min(max(__ldg(P.key_len + g.b), 0), P.n);
+                if (kv > 0) {
+                    int c_lo;
+                    slice_slots(P, g.s, (kv + kTileRows - 1) / kTileRows, c_lo, wslots);
                 }
+                if (w4 == 0)
+                    for (int j = lane; j < wslots; j += 32) poll_ge(P.wflag + (size_t)g.s * P.maxslots + j, 1, sAbort, P.status);
             }
             named_bar_sync(1 + grp, 128);
             if (*sAbort) ok = false;
@@ -1114,13 +1117,48 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             if (gtid < RP)
                 myG[gtid] = gtid < P.r ? (li < kMaxLoc ? sGc[li * 64 + gtid] : __ldcg(P.G + (size_t)idx * RP + gtid)) : neg_inf();
             if (g.phase == kPhaseOut) {
-                // stage W'^T (hi, lo) of this slice as the B operand: 128-byte rows, 16-byte chunks xor row%8
+                // W'^T = (Diag(beta)^-1 Gamma2 V)^T of this slice as the B operand (hi and lo parts; 128-byte rows =
+                // channels, 16-byte chunks of 8 pivots xor row % 8): every CTA of the slice adds the slots' partials
+                // itself, in slot order, so all of them hold the same bits
                 if (sego > 0 && ok) ok = wwait(bar(bWqEmpty), (sego - 1) & 1);
-                const uint4 *src = reinterpret_cast<const uint4 *>(P.Wb + (size_t)g.s * 2 * DK * 64);
-                for (int c = etid; c < 1024; c += kEpiThreads) {       // 1024 chunks of 16 bytes
-                    const int part = c >> 9, row = (c >> 3) & 63, ch = c & 7;
-                    const uint4 val = __ldcg(src + c);
-                    *reinterpret_cast<uint4 *>(smem + PL::offW + part * (DK * 128) + row * 128 + ((ch ^ (row & 7)) * 16)) = val;
+                const float mass = kv > 0 ? 1.f / (float)kv : 0.f;
+                for (int item = etid; item < DK * 8; item += kEpiThreads) {
+                    const int c = item >> 3, tc = item & 7, t0 = tc * 8;
+                    float acc8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    const float *src0 = P.wpart + (size_t)g.s * P.maxslots * (DK * 64) + c * 64 + t0;
+                    for (int sl0 = 0; sl0 < wslots; sl0 += 8) {
+                        float4 a[8], b[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            a[u] = b[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (sl0 + u < wslots) {
+                                const float4 *src = reinterpret_cast<const float4 *>(src0 + (size_t)(sl0 + u) * (DK * 64));
+                                a[u] = __ldcg(src);
+                                b[u] = __ldcg(src + 1);
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            acc8[0] += a[u].x; acc8[1] += a[u].y; acc8[2] += a[u].z; acc8[3] += a[u].w;
+                            acc8[4] += b[u].x; acc8[5] += b[u].y; acc8[6] += b[u].z; acc8[7] += b[u].w;
+                        }
+                    }
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int e2 = 0; e2 < 4; ++e2) {
+                        float wv2[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int t = t0 + e2 * 2 + u;
+                            wv2[u] = t < P.r ? acc8[e2 * 2 + u] * (mass / __ldg(P.beta + g.h * P.r + t)) : 0.f;
+                        }
+                        __nv_bfloat162 hh = __floats2bfloat162_rn(wv2[0], wv2[1]);
+                        hi[e2] = *reinterpret_cast<uint32_t *>(&hh);
+                        lo[e2] = pack_bf16(wv2[0] - __low2float(hh), wv2[1] - __high2float(hh));
+                    }
+                    uint8_t *dst = smem + PL::offW + c * 128 + ((tc ^ (c & 7)) * 16);
+                    *reinterpret_cast<uint4 *>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4 *>(dst + DK * 128) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
@@ -1232,12 +1270,15 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             else tiles(std::false_type{});
 
             if (g.phase == kPhaseWred) {
-                // ---- W accumulator of this segment: warp (qd, grp) takes its 32 lanes x 16 channels
+                // ---- W accumulator of this segment: TMEM lanes 0-63 hold the pivots' rows from the hi part of the plan,
+                // lanes 64-127 those from the lo part.  Warp (qd, grp < kWGroups) takes its 32 lanes x WC channels; the
+                // two halves are added through shared memory (the plan buffers are idle: every apply MMA has completed)
+                // and the CTA's partial goes to its slot, transposed to [channel][pivot].
+                constexpr int WC = DK / kWGroups;              // channels per reading group
+                float wv[WC];
                 if (ok) ok = wwait(bar(bWFull), segw & 1);
                 if (ok) {
-                    constexpr int WC = DK / kWGroups;              // channels per reading group
                     tc_fence_after();
-                    float wv[WC];
                     if (grp < kWGroups) {
                         tmem_ld<WC>(lane_addr + PL::colW + grp * WC, wv);
                         tmem_wait_ld();
@@ -1245,65 +1286,24 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(bWEmpty));
-                    if (grp < kWGroups) {
-                        float *dst = P.wpart + (((size_t)g.s * P.maxslots + g.slot) * 128 + rit) * DK + grp * WC;
-#pragma unroll
-                        for (int c = 0; c < WC; c += 4)
-                            __stcg(reinterpret_cast<float4 *>(dst + c), make_float4(wv[c], wv[c + 1], wv[c + 2], wv[c + 3]));
-                        __threadfence();
-                    }
                 }
                 ++segw;
-                named_bar_sync(5, kEpiThreads);
-                if (etid == 0) {
-                    __threadfence();
-                    const unsigned tk = atomicAdd(P.wticket + g.s, 1u);
-                    *sLastW = (tk == (unsigned)g.nslots - 1u) && !*sAbort;
+                float *xch = reinterpret_cast<float *>(smem + PL::offP);     // [channel][pivot] float
+                if (ok && grp < kWGroups && qd >= 2) {
+#pragma unroll
+                    for (int c = 0; c < WC; ++c) xch[(grp * WC + c) * 64 + rit - 64] = wv[c];
                 }
                 named_bar_sync(5, kEpiThreads);
-                if (*sLastW) {
+                if (ok && grp < kWGroups && qd < 2) {
+                    float *dst = P.wpart + ((size_t)g.s * P.maxslots + g.slot) * (DK * 64) + rit;
+#pragma unroll
+                    for (int c = 0; c < WC; ++c) __stcg(dst + (grp * WC + c) * 64, wv[c] + xch[(grp * WC + c) * 64 + rit]);
                     __threadfence();
-                    const float mass = g.nvalid > 0 ? 1.f / (float)g.nvalid : 0.f;
-                    // 64 pivots x 64 channels, four channels per thread; slots in order, four slots of loads in flight
-                    for (int e = etid; e < 64 * DK / 4; e += kEpiThreads) {
-                        const int tt = e / (DK / 4), c = (e % (DK / 4)) * 4;
-                        const float bt = tt < P.r ? __ldg(P.beta + g.h * P.r + tt) : 1.f;   // issued with the partial loads
-                        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-                        const float *src0 = P.wpart + ((size_t)g.s * P.maxslots * 128) * DK + c;
-                        for (int sl0 = 0; sl0 < g.nslots; sl0 += 6) {
-                            float4 a[6], b[6];
-#pragma unroll
-                            for (int u = 0; u < 6; ++u) {
-                                a[u] = b[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                if (sl0 + u < g.nslots) {
-                                    const float *src = src0 + ((size_t)(sl0 + u) * 128) * DK;
-                                    a[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)tt * DK));
-                                    b[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(64 + tt) * DK));
-                                }
-                            }
-#pragma unroll
-                            for (int u = 0; u < 6; ++u) {
-                                sum.x += a[u].x + b[u].x; sum.y += a[u].y + b[u].y;
-                                sum.z += a[u].z + b[u].z; sum.w += a[u].w + b[u].w;
-                            }
-                        }
-                        const float sc = tt < P.r ? mass / bt : 0.f;
-                        const float wv[4] = {sum.x * sc, sum.y * sc, sum.z * sc, sum.w * sc};
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const __nv_bfloat16 hi = __float2bfloat16_rn(wv[u]);
-                            const __nv_bfloat16 lo = __float2bfloat16_rn(wv[u] - __bfloat162float(hi));
-                            P.Wb[(((size_t)g.s * 2 + 0) * DK + c + u) * 64 + tt] = hi;
-                            P.Wb[(((size_t)g.s * 2 + 1) * DK + c + u) * 64 + tt] = lo;
-                        }
-                    }
+                }
+                named_bar_sync(5, kEpiThreads);
+                if (etid == 0 && !*sAbort) {
                     __threadfence();
-                    named_bar_sync(5, kEpiThreads);
-                    if (etid == 0) {
-                        __stcg(P.wticket + g.s, 0u);
-                        __threadfence();
-                        st_release(P.wdone + g.s, 1);
-                    }
+                    st_release(P.wflag + (size_t)g.s * P.maxslots + g.slot, 1);
                 }
             }
         }
@@ -1433,15 +1433,13 @@ FusedLayout fused_layout(int B, int H, int n, int d, int r)
     L.epoch = o; o += up256((size_t)2 * BH * 4);
     L.iter = o; o += up256((size_t)2 * BH * 4);
     L.robust = o; o += up256((size_t)2 * BH * 4);
-    L.wticket = o; o += up256((size_t)BH * 4);
-    L.wdone = o; o += up256((size_t)BH * 4);
+    L.wflag = o; o += up256((size_t)BH * ms * 4);
     L.gnat = o; o += up256((size_t)2 * BH * r * 4);
-    L.Wb = o; o += up256((size_t)BH * 2 * d * 64 * 2);
     L.part = o; o += up256((size_t)2 * 2 * BH * ms * RP * 2 * 8);
     L.head_end = o;
     L.kt = o; o += RP == 64 ? up256((size_t)2 * BH * ((n + 127) / 128) * 128 * 64 * 2) : 0;
     L.zprep = o; o += up256((size_t)H * 2 * RP * d * 2);
-    L.wpart = o; o += up256((size_t)BH * ms * 128 * d * 4);
+    L.wpart = o; o += up256((size_t)BH * ms * 64 * d * 4);
     L.total = o;
     return L;
 }
@@ -1489,9 +1487,7 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
     P.iter = reinterpret_cast<int *>(w + L.iter);
     P.robust = reinterpret_cast<int *>(w + L.robust);
     P.wpart = reinterpret_cast<float *>(w + L.wpart);
-    P.Wb = reinterpret_cast<__nv_bfloat16 *>(w + L.Wb);
-    P.wticket = reinterpret_cast<unsigned *>(w + L.wticket);
-    P.wdone = reinterpret_cast<int *>(w + L.wdone);
+    P.wflag = reinterpret_cast<int *>(w + L.wflag);
     P.out = static_cast<__nv_bfloat16 *>(out);
     P.g_nat = reinterpret_cast<float *>(w + L.gnat);
     P.status = reinterpret_cast<int *>(w + L.status);

@@ -64,7 +64,7 @@ cudaError_t launch_apply_out(const ApplyArgs &a, int dtype, cudaStream_t st);
 
 // ---- fused tensor-core path (lot_fused.cu): bf16 tensors, d = 64, r <= 64 ----
 struct FusedLayout {
-    size_t status, G, epoch, iter, robust, wticket, wdone, gnat, Wb, head_end, kt, zprep, part, wpart, total;
+    size_t status, G, epoch, iter, robust, wflag, gnat, head_end, kt, zprep, part, wpart, total;
 };
 bool fused_supported(int dtype, int d, int r);
 void fused_geometry(int B, int H, int n, int *q, int *ctas, int *maxslots, int *cps);
