@@ -44,9 +44,9 @@ namespace fused {
 using namespace sm100;
 
 constexpr int kPhaseSum = 0, kPhaseWred = 1, kPhaseOut = 2;
-constexpr int kGroups = 3;                        // epilogue groups of four warps (one per TMEM lane quarter)
+constexpr int kGroups = 2;                        // epilogue groups of four warps (one per TMEM lane quarter)
 constexpr int kEpiWarps = kGroups * 4;
-constexpr int kWGroups = kGroups == 4 ? 4 : 2;    // groups that read the W accumulator out (64 / kWGroups columns each)
+constexpr int kWGroups = kGroups == 4 ? 4 : (kGroups >= 2 ? 2 : 1);    // groups that read the W accumulator out (64 / kWGroups columns each)
 constexpr int kEpiThreads = kGroups * 128;
 constexpr int kThreads = 128 + kEpiThreads;        // warps 0-3: producer, MMA issuer, publisher, gatherer; then the epilogue
 constexpr int kMaxLoc = 16;                      // (slice, side) states of a CTA cached in shared memory
