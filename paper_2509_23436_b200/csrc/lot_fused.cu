@@ -15,9 +15,10 @@
 // tensor cores, W' = W / beta) and the OUT pass (query side: closing token update,
 // out = softmax-rows x W' on tensor cores).
 //
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 4-15 three epilogue
-// groups of 128 threads (tile k goes to group and TMEM accumulator k % 3), warp 2 the
-// publisher, warp 3 the gatherer.  Producer and MMA issuer never depend on G, so they run
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 4-11 kGroups = 2 epilogue
+// groups of 128 threads (tile k goes to group and TMEM accumulator k % kGroups), warp 2 the
+// publisher, warp 3 the gatherer.  (Two groups with 168 registers per thread measured faster than
+// three with 128.)  Producer and MMA issuer never depend on G, so they run
 // ahead across pass boundaries; only the epilogue warps wait, per segment, for the potential of
 // that attempt.
 //
@@ -54,6 +55,7 @@ constexpr int kTileRows = 128;
 constexpr int kDK = 64;                          // head dimension of this path
 constexpr int kStageBytes = kTileRows * kDK * 2; // one token tile: 128 rows x 64 bf16, 128-byte swizzled
 constexpr int kStages = 6;
+constexpr int kLock = 4;                         // rows of a stored-kernel tile a thread advances in step
 constexpr float kPlainFloor = 8.2718061e-25f;    // 2^-80: smallest column mass the plain sums may report
 
 struct alignas(64) FusedParams {
@@ -430,7 +432,6 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     constexpr uint32_t idesc_w = make_idesc_bf16(128, DK, 1, 1);
     constexpr uint32_t idesc_o = make_idesc_bf16(128, DK, 0, 0);
 
-    // The four service warps need few registers; give what they release to the sixteen epilogue warps.
     if (warp < 4) {
     if (warp == 0) {
         // ======================= TMA producer (one lane) =======================
@@ -528,7 +529,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         uint32_t gpar = 0;
         int ka = 0, ko = 0;                   // tiles of the apply passes / of the OUT pass so far
         bool ok = true, w_open = false;
-        // Apply MMAs are issued two tiles late, so that three tiles (one per epilogue group) are in flight:
+        // Apply MMAs are issued two tiles late, so that the logits of the following tiles are not held back by them:
         // pend_* is the older waiting tile, pnew_* the newer one.
         int pend_k = -1, pend_o = 0, pend_first = 0, pend_vs = 0, pend_phase = 0;
         int pnew_k = -1, pnew_o = 0, pnew_first = 0, pnew_vs = 0, pnew_phase = 0;
@@ -883,12 +884,12 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             if (ok) {
                                 const uint8_t *tile = smem + PL::offX + stg * kStageBytes;
 #pragma unroll
-                                for (int jp = 0; jp < 4; jp += 2) {
-                                    // two rows advance in step: every instruction has an independent twin
-                                    float2 kf[2][8], sa[2], sb[2];
-                                    float sr[2];
+                                for (int jp = 0; jp < 4; jp += kLock) {
+                                    // kLock rows advance in step: every instruction has independent twins
+                                    float2 kf[kLock][8], sa[kLock], sb[kLock];
+                                    float sr[kLock];
 #pragma unroll
-                                    for (int q = 0; q < 2; ++q) {
+                                    for (int q = 0; q < kLock; ++q) {
                                         const int rin = w4 * 32 + (jp + q) * 8 + rq;           // row inside the tile
                                         const uint4 a = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq) ^ (rin & 7)) * 16));
                                         const uint4 b = *reinterpret_cast<const uint4 *>(tile + rin * 128 + (((2 * cq + 1) ^ (rin & 7)) * 16));
@@ -901,28 +902,28 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
 #pragma unroll
                                     for (int e = 0; e < 8; e += 2) {
 #pragma unroll
-                                        for (int q = 0; q < 2; ++q) {
+                                        for (int q = 0; q < kLock; ++q) {
                                             sa[q] = __ffma2_rn(kf[q][e], w2[e], sa[q]);
                                             sb[q] = __ffma2_rn(kf[q][e + 1], w2[e + 1], sb[q]);
                                         }
                                     }
 #pragma unroll
-                                    for (int q = 0; q < 2; ++q) sr[q] = (sa[q].x + sa[q].y) + (sb[q].x + sb[q].y);
+                                    for (int q = 0; q < kLock; ++q) sr[q] = (sa[q].x + sa[q].y) + (sb[q].x + sb[q].y);
 #pragma unroll
-                                    for (int q = 0; q < 2; ++q) sr[q] += __shfl_xor_sync(0xffffffffu, sr[q], 1);
+                                    for (int q = 0; q < kLock; ++q) sr[q] += __shfl_xor_sync(0xffffffffu, sr[q], 1);
 #pragma unroll
-                                    for (int q = 0; q < 2; ++q) sr[q] += __shfl_xor_sync(0xffffffffu, sr[q], 2);
-                                    float2 uu[2];
+                                    for (int q = 0; q < kLock; ++q) sr[q] += __shfl_xor_sync(0xffffffffu, sr[q], 2);
+                                    float2 uu[kLock];
 #pragma unroll
-                                    for (int q = 0; q < 2; ++q) {
+                                    for (int q = 0; q < kLock; ++q) {
                                         const int rin = w4 * 32 + (jp + q) * 8 + rq;
                                         const float u = t * kTileRows + rin < g.nvalid ? __fdividef(1.f, sr[q]) : 0.f;
                                         uu[q] = make_float2(u, u);
                                     }
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) {
-                                        c2[e] = __ffma2_rn(kf[0][e], uu[0], c2[e]);
-                                        c2[e] = __ffma2_rn(kf[1][e], uu[1], c2[e]);
+#pragma unroll
+                                        for (int q = 0; q < kLock; ++q) c2[e] = __ffma2_rn(kf[q][e], uu[q], c2[e]);
                                     }
                                 }
                             }
@@ -1319,11 +1320,18 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
 
 // ---------------------------------------------------------------------------------------
 // Pivot preparation: Z' = Z * log2(e)/eps split into bf16 hi + lo, rows padded to RP with zeros.
-// Also raises LOT_DEV_EMPTY for non-positive key lengths.
+// Also clears the part of the workspace that must start at zero (`head`, head_vecs 16-byte words; the status word
+// lies before it and is cleared by block 0) and raises LOT_DEV_EMPTY for non-positive key lengths.
 // ---------------------------------------------------------------------------------------
 __global__ void zprep_kernel(const float *__restrict__ z, __nv_bfloat16 *__restrict__ zp, const int32_t *key_len,
-                             int *status, int B, int H, int r, int RP, int d, float scale)
+                             int *status, uint4 *head, size_t head_vecs, int B, int H, int r, int RP, int d, float scale)
 {
+    if (blockIdx.x == 0) {
+        if (threadIdx.x == 0) *status = 0;
+        __syncthreads();
+    }
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < head_vecs; i += (size_t)gridDim.x * blockDim.x)
+        head[i] = make_uint4(0u, 0u, 0u, 0u);
     const int total = H * RP * d;
     for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
         const int h = idx / (RP * d), rem = idx % (RP * d), t = rem / d, c = rem % d;
@@ -1469,7 +1477,6 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
     FusedLayout L = fused_layout(B, H, n, d, r);
     char *w = static_cast<char *>(ws);
     cudaError_t e;
-    if ((e = cudaMemsetAsync(ws, 0, L.head_end, st)) != cudaSuccess) return e;
 
     FusedParams P;
     memset(&P, 0, sizeof(P));
@@ -1499,7 +1506,13 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
 
     const float scale = (float)(1.4426950408889634 / (double)eps);
     const int total = H * RP * d;
-    zprep_kernel<<<(total + 255) / 256, 256, 0, st>>>(z, zp, key_len, P.status, B, H, r, RP, d, scale);
+    // the words after the 256-byte status block up to head_end must start at zero: the same kernel clears them
+    const size_t head_vecs = (L.head_end - 256) / 16;
+    int blocks = (int)((head_vecs + 255) / 256);
+    if (blocks < (total + 255) / 256) blocks = (total + 255) / 256;
+    if (blocks > 1184) blocks = 1184;
+    zprep_kernel<<<blocks, 256, 0, st>>>(z, zp, key_len, P.status, reinterpret_cast<uint4 *>(w + 256), head_vecs,
+                                         B, H, r, RP, d, scale);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
     if (RP == 16) e = launch_forward<16>(P, ctas, st);
