@@ -188,8 +188,8 @@ struct Plan {
     static constexpr int offMisc = offBar + 64 * 8;            // abort flag, TMEM base, flags
     static constexpr int offG = offMisc + 128;                 // float sG[kGroups][64]
     static constexpr int offGc = offG + kGroups * 64 * 4;      // float sGc[kMaxLoc][64]: this CTA's copy of the potentials
-    static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust, sMode [kMaxLoc]
-    static constexpr int offSeg = offState + 4 * kMaxLoc * 4;  // int sSeg[kMaxLoc][kSegInts]: static parts of the segments
+    static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust, sResFirst, sResLast [kMaxLoc]
+    static constexpr int offSeg = offState + 5 * kMaxLoc * 4;  // int sSeg[kMaxLoc][kSegInts]: static parts of the segments
     static constexpr int offWt = offSeg + kMaxLoc * kSegInts * 4; // float sWt[kMaxLoc][64]: weights 2^(G - max G) of the stored-kernel passes
     static constexpr int total = offWt + kMaxLoc * 64 * 4;
     // float sPart[2][kEpiWarps][64][2], the per-warp column pairs of the SUM passes, lives in the first plan buffer
@@ -361,13 +361,20 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     volatile int *sDone = reinterpret_cast<volatile int *>(smem + PL::offState);
     volatile int *sIter = sDone + kMaxLoc;
     volatile int *sRobust = sIter + kMaxLoc;
-    volatile int *sMode = sRobust + kMaxLoc;     // 1 = the next attempt reads the stored Gibbs kernel
+    // Attempts sResFirst[li] .. sResLast[li] of a segment read the stored Gibbs kernel (INT_MAX = not known yet).  There is
+    // one such run per segment, and both ends are written before the attempt they first matter for is released, so a
+    // warp that asks late about an old attempt (the MMA issuer has nothing to do in these passes) still gets that
+    // attempt's answer.
+    volatile int *sResFirst = sRobust + kMaxLoc;
+    volatile int *sResLast = sResFirst + kMaxLoc;
     volatile int *sPubDone = reinterpret_cast<volatile int *>(smem + PL::offMisc + 12);
     int *sSeg = reinterpret_cast<int *>(smem + PL::offSeg);
     // Wait until `need` attempts of local segment li (global index idx) are complete: 0 = gave up, else
     // 1 + robust flag + 2 * (the attempt reads the stored Gibbs kernel)
     auto seg_state = [&](int li, int idx, int need) -> int {
-        if (li < kMaxLoc) return spin_ge(sDone + li, need, sAbort, P.status) ? 1 + sRobust[li] + 2 * sMode[li] : 0;
+        if (li < kMaxLoc)
+            return spin_ge(sDone + li, need, sAbort, P.status)
+                       ? 1 + sRobust[li] + 2 * (need >= sResFirst[li] && need <= sResLast[li] ? 1 : 0) : 0;
         return poll_ge(P.epoch + idx, need, sAbort, P.status) ? 1 + __ldcg(P.robust + idx) : 0;
     };
     auto bar = [&](int id) { return smem_u32(bars + id); };
@@ -407,7 +414,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     }
     if (warp == 1) { tmem_alloc(smem_u32(sTmem), PL::tmem_cols); tmem_relinquish(); }
     for (int i = threadIdx.x; i < kMaxLoc * 64; i += kThreads) sGc[i] = 0.f;
-    if (threadIdx.x < 4 * kMaxLoc) sDone[threadIdx.x] = 0;
+    if (threadIdx.x < 3 * kMaxLoc) sDone[threadIdx.x] = 0;
+    else if (threadIdx.x < 5 * kMaxLoc) sDone[threadIdx.x] = 0x7fffffff;
     if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxLoc) {
         // segment table: one thread per (slice, side) of this CTA
         const int li = threadIdx.x - 128;
@@ -794,7 +802,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, off));
                 gmn = fminf(gmn, __shfl_xor_sync(0xffffffffu, gmn, off));
             }
-            const int next_resident = RP == 64 && cached && !fail && !rb && P.Kt != nullptr && (gmx - gmn) <= 64.f;
+            const bool run_started = cached && sResFirst[li] != 0x7fffffff, run_ended = cached && sResLast[li] != 0x7fffffff;
+            const int next_resident = RP == 64 && cached && !fail && !rb && !run_ended && P.Kt != nullptr && (gmx - gmn) <= 64.f;
             if (next_resident && mine) {
                 // weights of the next attempt, w_t = 2^(G_t - max G), computed once here for all epilogue warps
                 float *sWt = reinterpret_cast<float *>(smem + PL::offWt) + li * 64;
@@ -805,7 +814,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 __threadfence_block();
                 __syncwarp();
                 if (lane == 0) {
-                    sMode[li] = next_resident;
+                    if (next_resident && !run_started) sResFirst[li] = g.attempt + 1;
+                    if (!next_resident && run_started && !run_ended) sResLast[li] = g.attempt;
                     if (fail) sRobust[li] = 1;
                     else sIter[li] = itn + 1;
                     __threadfence_block();
