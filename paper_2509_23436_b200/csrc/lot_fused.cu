@@ -596,6 +596,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 if ((go - 1) >> 1) {                     // the epilogue reads the stored Gibbs kernel: nothing to issue
                     kx += g.t1 - g.t0;
                     k += g.t1 - g.t0;
+                    // This warp has not seen the fills of this segment complete, so it may not wait on a stage barrier by
+                    // parity again before they all have: wait until the segment has been gathered (every tile of it has
+                    // then been read).
+                    int done = 0;
+                    if (lane == 0) done = seg_state(g.li, idx, g.attempt + 1);
+                    done = __shfl_sync(0xffffffffu, done, 0);
+                    if (done == 0) { ok = false; break; }
                     continue;
                 }
             }
@@ -886,8 +893,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                                 c2[2 * j + 1] = make_float2(0.f, 0.f);
                             }
                         }
-                        // tile t0 + j goes to group j % kGroups: step straight from own tile to own tile
-                        for (int t = g.t0 + grp; t < g.t1; t += kGroups) {
+                        // A ring stage is always read by the same group (stage % kGroups; kStages is a multiple of kGroups),
+                        // whatever the segment: a parity wait on a stage's barrier is only safe for a waiter that has
+                        // itself seen the stage's previous fill complete.  (With the tile's index in the segment deciding
+                        // the group, a group could ask for fill f of a stage while fill f - 1, the other group's, was still
+                        // in flight, and the parity of fill f - 2 answered.)
+                        static_assert(kStages % kGroups == 0, "a ring stage must always fall to the same epilogue group");
+                        for (int t = g.t0 + (grp - kx % kGroups + kGroups) % kGroups; t < g.t1; t += kGroups) {
                             const int kxt = kx + (t - g.t0);
                             const int stg = kxt % kStages;
                             if (ok) ok = wwait(bar(bXFull + stg), (kxt / kStages) & 1);
