@@ -851,15 +851,18 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         float *myG = sG + grp * 64;
         Sched it(P, sSeg);
         Seg g;
-        int k = 0, ka = 0, ko = 0, segw = 0, sego = 0, segs = 0;
+        int k = 0;
         int gk = 0;                           // group of tile k
-        int kx = 0;                           // ring stage counter, as in the producer
         uint32_t mypar = 0;                   // parity of the number of tiles this group has taken
         bool ok = true;
-
-        while (it.next(g)) {
-            const int idx = g.side * BH + g.s;
-            if (g.phase == kPhaseSum) {
+        // The schedule lists every SUM segment before the first WRED segment: two loops, so that the state of one kind
+        // of pass is not carried through the other.
+        bool more = it.next(g);
+        {
+            int segs = 0;
+            int kx = 0;                       // ring stage counter, as in the producer
+            for (; more && g.phase == kPhaseSum; more = it.next(g)) {
+                const int idx = g.side * BH + g.s;
                 // ================= SUM: quad layout, column sums in registers =================
                 // every warp waits by itself for the potential of this attempt
                 const int li = g.li;
@@ -1113,9 +1116,12 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 };
                 if (rb) run(std::true_type{});
                 else run(std::false_type{});
-                continue;
             }
+        }
 
+        int ka = 0, ko = 0, segw = 0, sego = 0;
+        for (; more; more = it.next(g)) {
+            const int idx = g.side * BH + g.s;
             // ---- WRED / OUT: wait until the final potential (and W') of this slice is known here
             const int li = g.li;
             if (gtid == 0) {
@@ -1285,7 +1291,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             {
                 const int nt = g.t1 - g.t0;
                 gk = (gk + nt) % kGroups;
-                k += nt; ka += nt; kx += WRED ? 2 * nt : nt;
+                k += nt; ka += nt;
                 if (!WRED) ko += nt;
             }
             };
