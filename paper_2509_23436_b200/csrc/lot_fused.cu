@@ -62,6 +62,7 @@ struct alignas(64) FusedParams {
     CUtensorMap tmQ, tmK, tmV;   // [BH][n][64] bf16, box 64 x 128 x 1
     CUtensorMap tmZ;             // [2H][RP][64] bf16 (hi, lo of scaled pivots), box 64 x RP x 1
     CUtensorMap tmKt;            // [2BH][npad][64] bf16 stored Gibbs kernel (r > 32 only), box 64 x 128 x 1
+    CUtensorMap tmKtS;           // the same tensor with box 64 x 32 x 1: a warp's rows of a tile, for the store
     const float *beta;           // [H][r]
     const int32_t *key_len;      // [B] or nullptr
     __nv_bfloat16 *Kt;           // [2][BH][npad][64]: 2^(L_it - rowmax_i L), written by the first pass, or nullptr
@@ -195,6 +196,10 @@ struct Plan {
     // float sPart[2][kEpiWarps][64][2], the per-warp column pairs of the SUM passes, lives in the first plan buffer
     // (free until the WRED pass; the epilogue waits for the publisher's last read before it writes a plan tile)
     static constexpr int offPart = offP;
+    // the second plan buffer is, in the first pass, where every epilogue warp stages its 32 rows of a stored-kernel
+    // tile (4 KB, 128-byte swizzled like the tile itself) for the TMA store
+    static constexpr int offKtStage = offP + PBYTES;
+    static_assert(kEpiWarps * 32 * 128 <= PBYTES, "staging of the stored kernel must fit a plan buffer");
     static constexpr int dyn_bytes = total + 1024;             // slack for 1024-byte alignment
     static constexpr int tmem_cols = 512;
     static constexpr int colW = 256;                           // W accumulator (WRED): 64 columns
@@ -410,7 +415,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         *sPubDone = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.tmQ); prefetch_tensormap(&P.tmK); prefetch_tensormap(&P.tmZ); prefetch_tensormap(&P.tmV);
-        if (P.Kt != nullptr) prefetch_tensormap(&P.tmKt);
+        if (P.Kt != nullptr) { prefetch_tensormap(&P.tmKt); prefetch_tensormap(&P.tmKtS); }
     }
     if (warp == 1) { tmem_alloc(smem_u32(sTmem), PL::tmem_cols); tmem_relinquish(); }
     for (int i = threadIdx.x; i < kMaxLoc * 64; i += kThreads) sGc[i] = 0.f;
@@ -989,6 +994,11 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         mypar ^= 1u;
                         if (!ok) continue;
                         tc_fence_after();
+                        if (!RB && store_kt) {
+                            // the store of the previous tile must have read the staging rows before they are rewritten
+                            if (lane == 0) bulk_wait_group_read0();
+                            __syncwarp();
+                        }
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
                             float v[2 * NC];
@@ -1037,12 +1047,27 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                                 }
                             }
                             if (!RB && store_kt) {
-                                // G = 0 in this pass, so the exponentials are the stored kernel's entries
-                                __nv_bfloat16 *kt = P.Kt + ((size_t)idx * P.npad + (size_t)t * kTileRows + qd * 32 + half * 16 + rq) * 64 + 2 * cq;
+                                // G = 0 in this pass, so the exponentials are the stored kernel's entries: staged in shared
+                                // memory (rows of 128 bytes, 16-byte chunks xor row % 8) and written by one TMA store per warp
+                                // row A = half * 16 + rq, row B = row A + 8: both have row % 8 == rq, so one swizzled
+                                // address per column block serves both (the xor is kept inside the loop on purpose: hoisted,
+                                // the sixteen addresses would cost sixteen registers for the whole pass)
+                                const uint32_t rowA = smem_u32(smem) + PL::offKtStage + ((threadIdx.x >> 5) - 4) * (32 * 128) +
+                                                      (half * 16 + rq) * 128 + (rq << 4) + cq * 4;
 #pragma unroll
                                 for (int rep = 0; rep < NC / 2; ++rep) {
-                                    *reinterpret_cast<uint32_t *>(kt + rep * 8) = pack_bf16(v[rep * 4 + 0], v[rep * 4 + 1]);
-                                    *reinterpret_cast<uint32_t *>(kt + 8 * 64 + rep * 8) = pack_bf16(v[rep * 4 + 2], v[rep * 4 + 3]);
+                                    uint32_t addr;
+                                    asm volatile("xor.b32 %0, %1, %2;" : "=r"(addr) : "r"(rowA), "r"(rep << 4));
+                                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(pack_bf16(v[rep * 4 + 0], v[rep * 4 + 1])) : "memory");
+                                    asm volatile("st.shared.b32 [%0 + 1024], %1;" ::"r"(addr), "r"(pack_bf16(v[rep * 4 + 2], v[rep * 4 + 3])) : "memory");
+                                }
+                                if (half == 1) {
+                                    fence_proxy_async_smem();
+                                    __syncwarp();
+                                    if (lane == 0) {
+                                        tma_store_3d(&P.tmKtS, smem_u32(smem) + PL::offKtStage + ((threadIdx.x >> 5) - 4) * (32 * 128), 0, t * kTileRows + ((threadIdx.x >> 5) & 3) * 32, idx);
+                                        bulk_commit_group();
+                                    }
                                 }
                             }
                             float sA = sA0 + sA1, sB = sB0 + sB1;
@@ -1081,7 +1106,10 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     // ---- warp partial: the 8 rows-lanes of every column quarter, left in shared memory
                     if constexpr (!RB && NC == 16) {
                         const int cb = quad_col_reduce16(acc, lane);
-                        if (store_kt) asm volatile("fence.proxy.async.global;" ::: "memory");
+                        if (store_kt) {                      // the stores of this warp are complete before the segment is handed over
+                            if (lane == 0) bulk_wait_group0();
+                            __syncwarp();
+                        }
                         if (ok) ok = wwait(bar(bSegEmpty + par), par_empty);
                         *reinterpret_cast<float4 *>(dstp + ((cb >> 1) * 8 + 2 * cq) * 2) = make_float4(0.f, acc[0], 0.f, acc[1]);
                         __syncwarp();
@@ -1101,7 +1129,6 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             }
                         }
                     }
-                    if (store_kt) asm volatile("fence.proxy.async.global;" ::: "memory");
                     if (ok) ok = wwait(bar(bSegEmpty + par), par_empty);
                     if (rq == 0) {
 #pragma unroll
@@ -1514,7 +1541,8 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
         return cudaErrorInvalidValue;
     P.npad = ((n + 127) / 128) * 128;
     P.Kt = (RP == 64 && iters > 1) ? reinterpret_cast<__nv_bfloat16 *>(w + L.kt) : nullptr;
-    if (P.Kt != nullptr && !make_map(&P.tmKt, P.Kt, 2 * BH, P.npad, 64, 128)) return cudaErrorInvalidValue;
+    if (P.Kt != nullptr && (!make_map(&P.tmKt, P.Kt, 2 * BH, P.npad, 64, 128) || !make_map(&P.tmKtS, P.Kt, 2 * BH, P.npad, 64, 32)))
+        return cudaErrorInvalidValue;
     P.beta = beta; P.key_len = key_len;
     P.G = reinterpret_cast<float *>(w + L.G);
     P.part = reinterpret_cast<unsigned long long *>(w + L.part);
