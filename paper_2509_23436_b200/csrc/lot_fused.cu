@@ -538,7 +538,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         Sched it(P, sSeg);
         Seg g;
         int k = 0, kx = 0, ztag[2] = {-1, -1}, zuse[2] = {0, 0}, segw = 0, sego = 0;
-        int gk = 0;                           // group of tile k, and per-group tile-count parities
+        int gk = 0;                           // group of the next tile of the apply passes; per-group tile-count parities
         uint32_t gpar = 0;
         int ka = 0, ko = 0;                   // tiles of the apply passes / of the OUT pass so far
         bool ok = true, w_open = false;
@@ -637,10 +637,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             }
             const uint32_t za = dK_lo + ((PL::offZ + zs * PL::ZBYTES) >> 4);
             for (int t = g.t0; t < g.t1 && ok; ++t, ++k) {
-                const int grp = gk;                         // tile k goes to group k % kGroups
+                // SUM passes: the group is the ring stage's (stage % kGroups), as in the stored-kernel passes, so that a
+                // group has seen, through its accumulator, every earlier fill of a stage it later waits on by parity.
+                // Apply passes: the groups simply take turns.
+                const int grp = g.phase == kPhaseSum ? kx % kGroups : gk;
                 const uint32_t gbit = (gpar >> grp) & 1;    // parity of this group's tile count
                 gpar ^= 1u << grp;
-                gk = gk + 1 == kGroups ? 0 : gk + 1;
+                if (g.phase != kPhaseSum) gk = gk + 1 == kGroups ? 0 : gk + 1;
                 const int st = kx % kStages, ph = (kx / kStages) & 1;
                 ok = wwait2(bar(bXFull + st), ph, bar(bAccEmpty + grp), gbit ^ 1);
                 tc_fence_after();
@@ -857,7 +860,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
         Sched it(P, sSeg);
         Seg g;
         int k = 0;
-        int gk = 0;                           // group of tile k
+        int gk = 0;                           // group of the next tile of the apply passes
         uint32_t mypar = 0;                   // parity of the number of tiles this group has taken
         bool ok = true;
         // The schedule lists every SUM segment before the first WRED segment: two loops, so that the state of one kind
@@ -987,8 +990,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                         acc[ci] = 0.f;
                         if (RB) kap[ci] = neg_inf();
                     }
-                    // tile k goes to group k % kGroups: step straight from own tile to own tile
-                    const int first = grp >= gk ? grp - gk : grp - gk + kGroups;
+                    // the tile in ring stage st goes to group st % kGroups: step straight from own tile to own tile
+                    const int first = (grp - kx % kGroups + kGroups) % kGroups;
                     for (int t = g.t0 + first; t < g.t1; t += kGroups) {
                         if (ok) ok = wwait(bar(bAccFull + grp), mypar);
                         mypar ^= 1u;
@@ -1100,7 +1103,6 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                             }
                         }
                     }
-                    gk = (gk + (g.t1 - g.t0)) % kGroups;
                     k += g.t1 - g.t0;
                     kx += g.t1 - g.t0;
                     // ---- warp partial: the 8 rows-lanes of every column quarter, left in shared memory
