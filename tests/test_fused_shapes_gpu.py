@@ -51,3 +51,30 @@ def test_fused_path_matches_oracle(case):
         scale = max(1.0, np.abs(g1).max(), np.abs(g2).max())
         assert np.abs(res["g1"][b, h] - g1).max() <= 1e-3 * scale
         assert np.abs(res["g2"][b, h] - g2).max() <= 1e-3 * scale
+
+
+MIXED = [
+    # H, n, iters, scale of q, scale of k: scaled tokens widen the spread of that side's potentials, so that one side of
+    # a slice leaves the stored-kernel passes (spread above 64 binades) while the other stays on them
+    (4, 3000, 8, 8.0, 1.0),
+    (4, 3000, 8, 1.0, 8.0),
+    (16, 16384, 10, 8.0, 1.0),
+    (3, 2500, 9, 6.0, 6.0),
+]
+
+
+@pytest.mark.parametrize("case", MIXED, ids=lambda c: "H%d-n%d-T%d-q%g-k%g" % c)
+def test_fused_path_mixed_pass_kinds(case):
+    import dataclasses
+    H, n, iters, qs, ks = case
+    x = synth.make(1, H, n, 64, 64, seed=11, dtype=torch.bfloat16, eps=0.1, iters=iters)
+    x = dataclasses.replace(x, q=(x.q.float() * qs).to(torch.bfloat16), k=(x.k.float() * ks).to(torch.bfloat16))
+    res = gpu_forward(x, want_g=True)
+    assert res["status"] == 0
+    assert np.isfinite(res["out"]).all()
+    for h in sorted({0, H - 1}):
+        ref, g1, g2 = oracle_slice(x, 0, h, return_potentials=True)
+        assert head_err(res["out"][0, h], ref) <= 2e-2
+        scale = max(1.0, np.abs(g1).max(), np.abs(g2).max())
+        assert np.abs(res["g1"][0, h] - g1).max() <= 1e-3 * scale
+        assert np.abs(res["g2"][0, h] - g2).max() <= 1e-3 * scale
