@@ -1,36 +1,42 @@
 // Fused tensor-core path of the LOT attention forward for bf16 tensors (sm_100a): ONE persistent,
 // cooperatively launched kernel runs every Sinkhorn pass and both apply stages.
 //
-// The similarity matrices are never stored: every pass recomputes the logits of a 128-token
-// tile with tcgen05.mma (bf16 tokens x pivots pre-scaled by log2(e)/eps and split into bf16
-// hi + lo parts, f32 accumulation in TMEM), tokens staged by TMA.  With the token potential
-// eliminated the state of a solve (Eq. (1)-(2), scaling form) is the pivot potential G:
+// The n x r similarity matrices are never stored as such.  The first Sinkhorn pass, and every pass of
+// a solve that cannot use the stored kernel (r <= 32, potentials spread over more than 64 binades, a
+// column sum that underflowed), recomputes the logits of a 128-token tile with tcgen05.mma (bf16
+// tokens x pivots pre-scaled by log2(e)/eps and split into bf16 hi + lo parts, f32 accumulation in
+// TMEM), tokens staged by TMA.  For 32 < r <= 64 the first pass keeps 2^(L - rowmax), the stabilised
+// Gibbs kernel of the scaling form of Eq. (1)-(2), as bf16 (staged in shared memory, one TMA store per
+// warp and tile); the later passes stream it back and are the paper's matrix-vector scalings.  With
+// the token potential eliminated the state of a solve is the pivot potential G:
 //   token update : row log-sum-exp over the pivots (inside a thread quad / a thread)
 //   pivot update : column sums over the tokens of the row-normalised tile, per (slice, side)
 //
-// Work split.  CTA c owns tiles [c*q, (c+1)*q) of the slice-major tile list, for both sides, in
-// every pass; a (slice, side) range of it is a segment.  Pass order: T SUM passes (both sides,
-// one pivot update each), one spare SUM pass for segments that had to repeat an update with
-// (kappa, S) column pairs, the WRED pass (key side: closing token update, W = Gamma2 V on
-// tensor cores, W' = W / beta) and the OUT pass (query side: closing token update,
-// out = softmax-rows x W' on tensor cores).
+// Work split.  CTA c owns a fixed range of the slice-major tile list, for both sides, in every pass
+// (with few slices: the same number of CTAs per slice, none spanning two); a (slice, side) range of it
+// is a segment.  Pass order: T SUM passes (both sides, one pivot update each), one spare SUM pass for
+// segments that had to repeat an update with (kappa, S) column pairs, the WRED pass (key side: closing
+// token update, W = Gamma2 V on tensor cores) and the OUT pass (query side: closing token update,
+// out = softmax-rows x W' on tensor cores, W' = W / beta).
 //
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 4-11 kGroups = 2 epilogue
-// groups of 128 threads (tile k goes to group and TMEM accumulator k % kGroups), warp 2 the
-// publisher, warp 3 the gatherer.  (Two groups with 168 registers per thread measured faster than
-// three with 128.)  Producer and MMA issuer never depend on G, so they run
-// ahead across pass boundaries; only the epilogue warps wait, per segment, for the potential of
-// that attempt.
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warp 2 the publisher, warp 3 the
+// gatherer, warps 4-11 kGroups = 2 epilogue groups of 128 threads (two groups with 168 registers per
+// thread measured faster than three with 128).  In the SUM passes the tile in ring stage st belongs to
+// group st % kGroups: the epilogue waits on a stage's barrier by parity, which is only valid for a
+// waiter that has seen the stage's previous fill complete.  In the apply passes the groups take turns.
+// Producer and MMA issuer never depend on G, so they run ahead across pass boundaries; only the
+// epilogue warps wait, per segment, for the potential of that attempt.
 //
-// Cross-CTA protocol (all CTAs are co-resident: cooperative launch, one CTA per SM).  The
-// epilogue warps leave their column partials of a segment in shared memory and go on; the
-// publisher warp adds them in warp order and writes the CTA's partial to its slot as 64-bit
-// words that carry the attempt number beside the value, so a word is valid by itself and no
-// fence or ticket is needed.  The gatherer warp of EVERY CTA that shares the (slice, side) polls
-// all slots until their tags match, merges them in slot order (deterministic and identical in
-// all CTAs, including the verdict that plain sums underflowed), updates its copy of G and hands
-// it to its epilogue warps through shared memory.  Every wait, on an mbarrier, on shared or on
-// global memory, is bounded in time and raises LOT_DEV_TIMEOUT.
+// Cross-CTA protocol (all CTAs are co-resident: cooperative launch, one CTA per SM).  The epilogue
+// warps leave their column partials of a segment in shared memory and go on; the publisher warp adds
+// them in warp order and writes the CTA's partial to its slot as 64-bit words that carry the attempt
+// number beside the value, so a word is valid by itself and no fence or ticket is needed.  The
+// gatherer warp of EVERY CTA that shares the (slice, side) polls all slots until their tags match,
+// merges them in slot order (deterministic and identical in all CTAs, including the verdict that
+// plain sums underflowed), updates its copy of G and hands it to its epilogue warps through shared
+// memory.  W is merged the same way: every CTA writes its partial to its slot and raises a flag, and
+// every CTA of the slice adds the slots itself, in slot order.  Every wait, on an mbarrier, on shared
+// or on global memory, is bounded in time and raises LOT_DEV_TIMEOUT.
 #include "lot_common.cuh"
 #include "lot_internal.h"
 #include "lot_sm100.cuh"
