@@ -246,7 +246,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the call (all its kernels together; see the design doc for the byte model)
+    # ---- roofline of the call (all its kernels together): algorithmic bytes = Q, K, V read once, out written once, pivots
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(peaks_path):
         peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
