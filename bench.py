@@ -37,12 +37,20 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--n", type=int, default=16384)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    return ap.parse_args()
+    ap.add_argument("--iters", type=int, default=None,
+                    help="Sinkhorn iterations (default: the configuration's 10); for profiling single phases, e.g. 0 = apply passes only")
+    args = ap.parse_args()
+    global ITERS
+    ITERS = args.iters
+    return args
+
+
+ITERS = None
 
 
 def workload(n, rank=0):
     from paper_2509_23436_b200 import synth
-    return synth.config(4, n=n, variant=rank)
+    return synth.config(4, n=n, variant=rank, iters=ITERS)
 
 
 def algorithmic_bytes(B, H, n, d, r, s_in, s_out):
@@ -258,7 +266,7 @@ def run_ours(args):
     per_call_ms = sum(times) / len(times)
     achieved = abytes / (per_call_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": 251.2e6 if (n == 16384 and fused) else None, "peak_source": peak_src,
+                "traffic": 251.2e6 if (n == 16384 and fused and ITERS is None) else None, "peak_source": peak_src,
                 "algorithmic_bytes": abytes,
                 "kernel": "fused_forward_kernel (persistent; the call is this kernel plus a 3 us pivot preparation)"
                           if fused else "whole lot_attention_fwd_ex call (all launches)"}
