@@ -1,5 +1,5 @@
 // Thin wrappers over the sm_100a instructions the fused kernels use: mbarrier, TMA tensor
-// loads (no multicast), tcgen05 tensor-core MMA with TMEM accumulators, TMEM loads.
+// loads (into the issuing CTA's shared memory only), tcgen05 tensor-core MMA with TMEM accumulators, TMEM loads.
 // Every wait is bounded: it gives up after about kWaitLimitNs of wall time, raises the CTA's
 // abort flag and the caller-visible LOT_DEV_TIMEOUT status bit, and returns false.
 #pragma once
@@ -82,7 +82,7 @@ __device__ __forceinline__ void fence_proxy_async_smem()
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// ---- TMA (tiled tensor loads into this CTA's shared memory; never multicast) ------------
+// ---- TMA (tiled tensor loads into this CTA's shared memory) -----------------------------------
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2)
 {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
