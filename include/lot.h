@@ -152,10 +152,11 @@ LOT_API size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype)
  * parameters launches (host arithmetic only; 0 for iters < 0).  bf16 tensors with d = 64 and
  * r <= 64 take the fused tensor-core path: one persistent kernel for all passes (launched
  * cooperatively: it needs as many free SMs as it has thread blocks, at most one per SM) plus a
- * small pivot preparation, which also clears the part of the workspace that must start at zero.  For 32 < r <= 64 its first pass keeps the stabilised Gibbs kernel
- * exp(C/eps - rowmax) of both sides as bf16 in the workspace and the later passes iterate on
- * that copy (potentials then agree with an exact float evaluation to about 1e-4, the output
- * to the bf16 rounding of `out`).  Every other supported shape takes the general path.
+ * small pivot preparation, which also clears the part of the workspace that must start at
+ * zero.  For 32 < r <= 64 its first pass keeps the stabilised Gibbs kernel exp(C/eps - rowmax)
+ * of both sides as bf16 in the workspace and the later passes iterate on that copy (potentials
+ * then agree with an exact float evaluation to about 1e-4, the output to the bf16 rounding of
+ * `out`).  Every other supported shape takes the general path.
  */
 LOT_API int lot_launch_count(int dtype, int d, int r, int iters);
 
