@@ -5,8 +5,8 @@
  * For each (batch b, head h) slice, with queries/keys/values q,k,v [n,d], pivot
  * locations z_h [r,d] and pivot masses beta_h [r] (> 0, summing to 1):
  *
- *   costs        C1[i,t] = <q_i, z_t>,  C2[j,t] = <k_j, z_t>            (display after
- *                "Setting similarity to c(q,k) = q^T k"; no 1/sqrt(d) factor)
+ *   costs        C1[i,t] = <q_i, z_t>,  C2[j,t] = <k_j, z_t>            (Section "Method", the
+ *                unnumbered display defining C^(1), C^(2) before Eq. (1); no 1/sqrt(d) factor)
  *   two solves   Gamma1 in U(beta, a), Gamma2 in U(beta, b), the entropic problems
  *                Eq. (1)-(2), in the Sinkhorn scaling form Diag(u) exp(C/eps) Diag(v)
  *   composition  Gamma = Gamma1^T Diag(beta)^-1 Gamma2 (Eq. (3)), never formed
@@ -88,7 +88,8 @@ LOT_API const char *lot_status_string(int status);
 /*
  * lot_cost -- the similarity matrices of Section "Method": cost[b,h,i,t] = <x[b,h,i,:], z[h,t,:]>.
  *   x     [B,H,n,d] in `dtype`;  z [H,r,d] float32;  cost [B,H,n,r] float32 (out).
- * float32 accumulation; bf16 inputs are used exactly.  Needs no workspace.
+ * bf16 inputs are used exactly and accumulate in float32; float32 inputs accumulate in float64
+ * and the result is rounded to float32 once.  Needs no workspace.
  */
 LOT_API int lot_cost(const void *x, const float *z, int dtype, int B, int H, int n, int d, int r,
              float *cost, lot_stream_t stream);
@@ -148,17 +149,22 @@ LOT_API int lot_sinkhorn_static(const float *cost, const float *beta, const int3
 LOT_API size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype);
 
 /*
- * lot_launch_count -- how many kernels of this library one lot_attention_fwd_ex call with these
- * parameters launches (host arithmetic only; 0 for iters < 0).  bf16 tensors with d = 64 and
- * r <= 64 take the fused tensor-core path: one persistent kernel for all passes (launched
- * cooperatively: it needs as many free SMs as it has thread blocks, at most one per SM) plus a
- * small pivot preparation, which also clears the part of the workspace that must start at
- * zero.  For 32 < r <= 64 its first pass keeps the stabilised Gibbs kernel exp(C/eps - rowmax)
- * of both sides as bf16 in the workspace and the later passes iterate on that copy (potentials
+ * lot_path -- which implementation one lot_attention_fwd_ex call with these parameters takes (host
+ * arithmetic only): 0 = the general path (a cost kernel per side, one kernel per Sinkhorn pass, two
+ * apply kernels), 1 = the fused tensor-core path (bf16 tensors, d = 64, r <= 64: one persistent
+ * kernel for all passes, launched cooperatively, plus a small pivot preparation).  On the fused
+ * path with 32 < r <= 64 the first pass keeps the stabilised Gibbs kernel exp(C/eps - rowmax) of
+ * the scaling form of Eq. (1)-(2) as bf16 and the later passes iterate on that copy (potentials
  * then agree with an exact float evaluation to about 1e-4, the output to the bf16 rounding of
- * `out`).  Every other supported shape takes the general path.
+ * `out`).
  */
-LOT_API int lot_launch_count(int dtype, int d, int r, int iters);
+LOT_API int lot_path(int dtype, int B, int H, int n, int d, int r, int iters);
+
+/*
+ * lot_launch_count -- how many kernels of this library one lot_attention_fwd_ex call with these
+ * parameters launches (host arithmetic only; 0 for iters < 0).
+ */
+LOT_API int lot_launch_count(int dtype, int B, int H, int n, int d, int r, int iters);
 
 /*
  * lot_attention_fwd_ex -- the whole forward path, Eq. (1)-(4): costs, both solves, apply.

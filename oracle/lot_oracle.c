@@ -37,7 +37,7 @@
 #include <omp.h>
 #endif
 
-/* ---- Section "Method", display after "Setting similarity to c(q,k)=q^T k":
+/* ---- Section "Method", the unnumbered display that defines C^(1), C^(2) before Eq. (1):
  *      C_it = z_t^T x_i. */
 void lot_oracle_cost(const double *x, const double *z, int n, int d, int r, double *C)
 {
@@ -181,7 +181,7 @@ void lot_oracle_head(const double *q, const double *k, const double *v,
 }
 
 /* ---- All (batch, head) slices.  q,k,v,out [B,H,n,d]; z [H,r,d]; beta [H,r]
- *      (per head, shared over the batch: "each head has its own (Z, sigma)").
+ *      (per head, shared over the batch: Section "Method", closing remark on multi-head attention).
  *      Query marginal uniform 1/n.  Key marginal uniform 1/n, or, when
  *      key_len != NULL, 1/key_len[b] on tokens j < key_len[b] and zero beyond.
  *      g1,g2 [B,H,r] optional.  Slices are independent; OpenMP runs them side

@@ -31,7 +31,8 @@ SIGNATURES = {
     "lot_sinkhorn": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lot_sinkhorn_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _vp]),
     "lot_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
-    "lot_launch_count": (_i, [_i, _i, _i, _i]),
+    "lot_path": (_i, [_i, _i, _i, _i, _i, _i, _i]),
+    "lot_launch_count": (_i, [_i, _i, _i, _i, _i, _i, _i]),
     "lot_attention_fwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
                                   _vp, _vp, _vp, _vp, _sz, _vp]),
     "lot_attention_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp]),
@@ -147,8 +148,12 @@ def lot_workspace_bytes(B, H, n, d, r, dtype_code) -> int:
     return lib().lot_workspace_bytes(B, H, n, d, r, dtype_code)
 
 
-def lot_launch_count(dtype_code: int, d: int, r: int, iters: int) -> int:
-    return lib().lot_launch_count(dtype_code, d, r, iters)
+def lot_path(dtype_code: int, B: int, H: int, n: int, d: int, r: int, iters: int) -> int:
+    return lib().lot_path(dtype_code, B, H, n, d, r, iters)
+
+
+def lot_launch_count(dtype_code: int, B: int, H: int, n: int, d: int, r: int, iters: int) -> int:
+    return lib().lot_launch_count(dtype_code, B, H, n, d, r, iters)
 
 
 def lot_attention_fwd_ex(q, k, v, z, beta, key_len, eps, iters, *, out=None, g1_out=None, g2_out=None,

@@ -181,10 +181,16 @@ int lot_sinkhorn_static(const float *cost, const float *beta, const int32_t *len
                         float *g, float *f, float *plan, int32_t *status_out,
                         lot_stream_t stream)
 {
+    // every argument check comes first, in lot_sinkhorn's order, so that a bad call is refused before any device work
     int st = check_dims(B, H, n, r);
     if (st != LOT_OK) return st;
+    if (!(eps > 0.f) || !isfinite(eps) || iters < 0) return LOT_ERR_INVALID_ARG;
     if (status_out && (reinterpret_cast<uintptr_t>(status_out) & 3u)) return LOT_ERR_INVALID_ARG;
     if (B == 0 || n == 0) return LOT_OK;
+    if (!cost || !beta || !g) return LOT_ERR_INVALID_ARG;
+    if (!aligned16(cost) || !aligned16(beta) || !aligned16(g) || !aligned16(f) || !aligned16(plan) ||
+        (len && (reinterpret_cast<uintptr_t>(len) & 3u)))
+        return LOT_ERR_INVALID_ARG;
     if (sink_layout(B * H, n, r, 0, 8).total > (size_t)LOT_STATIC_SCRATCH_BYTES) return LOT_ERR_WORKSPACE;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LOT_ERR_CUDA;
@@ -217,10 +223,16 @@ size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype)
     return attn_layout(B, H, n, d, r, dtype).total;
 }
 
-int lot_launch_count(int dtype, int d, int r, int iters)
+int lot_path(int dtype, int B, int H, int n, int d, int r, int iters)
+{
+    (void)B; (void)H; (void)n; (void)iters;
+    return fused_supported(dtype, d, r) ? 1 : 0;
+}
+
+int lot_launch_count(int dtype, int B, int H, int n, int d, int r, int iters)
 {
     if (iters < 0) return 0;
-    if (fused_supported(dtype, d, r)) return fused_launches(iters);
+    if (lot_path(dtype, B, H, n, d, r, iters) != 0) return fused_launches(iters);
     return 2 + iters + 1 + 2;
 }
 

@@ -59,7 +59,41 @@ def worst_head_err(got, ref):
     return max(head_err(got[b, h], ref[b, h]) for b in range(B) for h in range(H))
 
 
-def elem_err(got, ref, tol):
-    """Elementwise relative error with the absolute floor tol * rms(ref) (reported, not gated)."""
-    floor = tol * float(np.sqrt((ref ** 2).mean()))
-    return float((np.abs(got - ref) / np.maximum(np.abs(ref), floor / tol)).max())
+def elem_err(got, ref):
+    """Elementwise relative error of one slice, max over entries of |got - ref| / max(|ref|, rms(ref)): entries
+    smaller than the slice's root mean square are measured against that floor (an absolute error of tol * rms),
+    so that a near-zero reference entry does not decide the figure.  Gated at the same tolerance as head_err."""
+    floor = float(np.sqrt((ref ** 2).mean()))
+    return float((np.abs(got - ref) / np.maximum(np.abs(ref), floor)).max())
+
+
+def check_slice(got, ref, tol, what=""):
+    """Both error figures of one (batch, head) slice against the tolerance; returns them."""
+    he, ee = head_err(got, ref), elem_err(got, ref)
+    assert he <= tol, f"{what}: normwise error {he:.3e} > {tol}"
+    assert ee <= tol, f"{what}: elementwise error {ee:.3e} > {tol} (normwise {he:.3e})"
+    return he, ee
+
+
+def oracle_slices(x, slices, return_potentials=False):
+    """Oracle results of several (batch, head) slices in one call (the oracle threads over slices)."""
+    d = x.f64()
+    bs = [b for b, _ in slices]
+    hs = [h for _, h in slices]
+    # one problem per requested slice: batch index runs over the list, one head each
+    outs, g1s, g2s = [], [], []
+    import concurrent.futures as cf
+
+    def one(bh):
+        b, h = bh
+        kl = None if d["key_len"] is None else d["key_len"][b:b + 1]
+        return O.attention_fwd(d["q"][b:b + 1, h:h + 1], d["k"][b:b + 1, h:h + 1], d["v"][b:b + 1, h:h + 1],
+                               d["z"][h:h + 1], d["beta"][h:h + 1], x.eps, x.iters, key_len=kl, threads=1,
+                               return_potentials=True)
+    with cf.ThreadPoolExecutor(max_workers=min(len(slices), 8)) as ex:
+        res = list(ex.map(one, list(zip(bs, hs))))
+    for o, g1, g2, _ in res:
+        outs.append(o[0, 0]); g1s.append(g1[0, 0]); g2s.append(g2[0, 0])
+    if return_potentials:
+        return outs, g1s, g2s
+    return outs

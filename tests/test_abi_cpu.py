@@ -38,7 +38,8 @@ def test_workspace_queries_are_host_only(L):
     assert 0 < L.lot_workspace_bytes(1, 16, 16384, 64, 64, lot.LOT_BF16) < a // 3
     # and nothing of size n x r for r <= 32
     assert 0 < L.lot_workspace_bytes(1, 16, 16384, 64, 32, lot.LOT_BF16) < a // 16
-    assert L.lot_launch_count(lot.LOT_BF16, 64, 64, 10) > 0 and L.lot_launch_count(lot.LOT_F32, 64, 64, 10) == 15
+    assert L.lot_launch_count(lot.LOT_BF16, 1, 16, 16384, 64, 64, 10) > 0
+    assert L.lot_launch_count(lot.LOT_F32, 1, 16, 16384, 64, 64, 10) == 15 and L.lot_path(lot.LOT_F32, 1, 16, 16384, 64, 64, 10) == 0
     assert L.lot_workspace_bytes(1, 16, 16384, 64, 300, lot.LOT_BF16) == 0      # r too large
     assert L.lot_workspace_bytes(1, 16, 16384, 60, 64, lot.LOT_BF16) == 0       # d % 8 != 0
     assert L.lot_sinkhorn_workspace_bytes(2, 3, 100, 16) > 0

@@ -7,7 +7,7 @@ import pytest
 import torch
 
 from paper_2509_23436_b200 import synth
-from lot_testutil import gpu_forward, head_err, oracle_slice
+from lot_testutil import check_slice, gpu_forward, oracle_slice
 
 pytestmark = pytest.mark.gpu
 
@@ -33,6 +33,13 @@ CASES = [
     (1, 7, 1500, 17, 5, 0.1, True),
     (1, 9, 1000, 8, 4, 0.1, False),
     (1, 37, 4096, 64, 3, 0.1, False),
+    # many short slices: ten and more (slice, side) pairs per thread block
+    (128, 12, 100, 64, 3, 0.1, False),
+    (512, 3, 197, 16, 4, 0.1, True),
+    (96, 4, 150, 64, 5, 0.01, False),
+    # the benchmark shapes of configs 2 and 3 at a training-size batch
+    (64, 3, 197, 16, 10, 0.1, False),
+    (32, 12, 512, 32, 20, 0.05, True),
 ]
 
 
@@ -46,7 +53,7 @@ def test_fused_path_matches_oracle(case):
     assert np.isfinite(res["out"]).all()
     for (b, h) in sorted({(0, 0), (B // 2, H // 2), (B - 1, H - 1)}):
         ref, g1, g2 = oracle_slice(x, b, h, return_potentials=True)
-        assert head_err(res["out"][b, h], ref) <= 2e-2
+        check_slice(res["out"][b, h], ref, 2e-2, f"slice {(b, h)}")
         # potentials: stored-kernel passes round the Gibbs kernel to bf16 once (see test_parity_gpu)
         scale = max(1.0, np.abs(g1).max(), np.abs(g2).max())
         assert np.abs(res["g1"][b, h] - g1).max() <= 1e-3 * scale
@@ -74,7 +81,7 @@ def test_fused_path_mixed_pass_kinds(case):
     assert np.isfinite(res["out"]).all()
     for h in sorted({0, H - 1}):
         ref, g1, g2 = oracle_slice(x, 0, h, return_potentials=True)
-        assert head_err(res["out"][0, h], ref) <= 2e-2
+        check_slice(res["out"][0, h], ref, 2e-2, f"head {h}")
         scale = max(1.0, np.abs(g1).max(), np.abs(g2).max())
         assert np.abs(res["g1"][0, h] - g1).max() <= 1e-3 * scale
         assert np.abs(res["g2"][0, h] - g2).max() <= 1e-3 * scale

@@ -31,7 +31,7 @@ def _uniform(n):
     return np.full(n, 1.0 / n)
 
 
-# ---------------------------------------------------------------- cost (display after "Setting similarity ...")
+# ---------------------------------------------------------------- cost (Section "Method", display defining C^(1), C^(2))
 def test_cost_is_plain_dot_product_no_scaling():
     q, _, _, z, _ = _rand_problem(n=7, d=6, r=3, seed=1)
     C = O.cost(q, z)

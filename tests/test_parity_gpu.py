@@ -9,7 +9,8 @@ from oracle import lot_oracle as O
 from paper_2509_23436_b200 import binding as lot
 from paper_2509_23436_b200 import synth
 
-from lot_testutil import TOL, gpu_forward, head_err, oracle_all, oracle_slice, to_dev, worst_head_err
+from lot_testutil import (TOL, check_slice, gpu_forward, head_err, oracle_all, oracle_slice, oracle_slices, to_dev,
+                          worst_head_err)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -86,8 +87,12 @@ def _check_full(x, want_g=True):
     d = x.f64()
     ref, g1, g2, _ = O.attention_fwd(d["q"], d["k"], d["v"], d["z"], d["beta"], x.eps, x.iters,
                                      key_len=d["key_len"], return_potentials=True)
-    err = worst_head_err(res["out"], ref)
-    assert err <= TOL[x.q.dtype], f"{x.name} {x.q.dtype}: {err}"
+    err, worst_elem = 0.0, 0.0
+    for b in range(ref.shape[0]):
+        for h in range(ref.shape[1]):
+            he, ee = check_slice(res["out"][b, h], ref[b, h], TOL[x.q.dtype], f"{x.name} {x.q.dtype} slice {(b, h)}")
+            err, worst_elem = max(err, he), max(worst_elem, ee)
+    print(f"{x.name} {x.q.dtype}: normwise {err:.3e}, elementwise {worst_elem:.3e}")
     if want_g:
         # potentials: float32 tensors 1e-4; bf16 tensors 1e-3, because passes 2..T of the fused bf16 path read the
         # Gibbs kernel exp(C/eps - rowmax) back as bf16 (relative rounding 2^-9 per entry, averaged over the tokens)
@@ -128,32 +133,42 @@ def test_config4_long_context_bf16_all_heads(n):
     _check_full(synth.config(4, n=n), want_g=False)
 
 
-def test_config4_n65536_sampled_heads():
+def test_config4_n65536_all_heads_and_potentials():
+    """The one length of config 4 whose stored Gibbs kernel (268 MB) does not stay in the L2."""
     x = synth.config(4, n=65536)
-    res = gpu_forward(x)
+    res = gpu_forward(x, want_g=True)
     assert res["status"] == 0
-    for h in (0, 7, 15):
-        assert head_err(res["out"][0, h], oracle_slice(x, 0, h)) <= 2e-2
+    H = x.shape[1]
+    outs, g1s, g2s = oracle_slices(x, [(0, h) for h in range(H)], return_potentials=True)
+    for h in range(H):
+        check_slice(res["out"][0, h], outs[h], 2e-2, f"n=65536 head {h}")
+        sc = max(1.0, np.abs(g1s[h]).max(), np.abs(g2s[h]).max())
+        assert np.abs(res["g1"][0, h] - g1s[h]).max() <= 1e-3 * sc
+        assert np.abs(res["g2"][0, h] - g2s[h]).max() <= 1e-3 * sc
 
 
 def test_config4_fp32_n4096():
     _check_full(synth.config(4, n=4096, dtype=torch.float32), want_g=False)
 
 
-# ----------------------------------------------------------------------------- config 5 (rank / iteration stress), sampled
-@pytest.mark.parametrize("r,iters,eps,dtype", [
-    (16, 5, 0.1, torch.bfloat16), (64, 20, 0.1, torch.bfloat16), (128, 5, 0.1, torch.bfloat16),
-    (256, 5, 0.1, torch.bfloat16), (64, 20, 0.01, torch.bfloat16), (256, 20, 0.01, torch.bfloat16),
-    (64, 50, 0.01, torch.float32), (16, 50, 0.1, torch.float32), (128, 20, 0.01, torch.float32),
-])
-def test_config5_stress_sampled_slices(r, iters, eps, dtype):
+# ----------------------------------------------------------------------------- config 5 (rank / iteration stress): the whole grid
+CFG5_SLICES = ((0, 0), (1, 3), (2, 5), (3, 7))
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32], ids=["bf16", "f32"])
+@pytest.mark.parametrize("eps", [0.1, 0.01])
+@pytest.mark.parametrize("iters", [5, 20, 50])
+@pytest.mark.parametrize("r", [16, 64, 128, 256])
+def test_config5_stress_grid(r, iters, eps, dtype):
+    """Every cell of config 5 (4 ranks x 3 iteration counts x 2 eps x 2 dtypes) at full size; the oracle checks four
+    (batch, head) slices of each, the first and the last among them, and every output entry must be finite."""
     x = synth.config(5, r=r, iters=iters, eps=eps, dtype=dtype)
     res = gpu_forward(x)
     assert res["status"] == 0
     assert np.isfinite(res["out"]).all()
-    for (b, h) in ((0, 0), (3, 7)):
-        err = head_err(res["out"][b, h], oracle_slice(x, b, h))
-        assert err <= TOL[dtype], f"r={r} T={iters} eps={eps} {dtype} slice {(b, h)}: {err}"
+    refs = oracle_slices(x, CFG5_SLICES)
+    for (b, h), ref in zip(CFG5_SLICES, refs):
+        check_slice(res["out"][b, h], ref, TOL[dtype], f"r={r} T={iters} eps={eps} {dtype} slice {(b, h)}")
 
 
 # ----------------------------------------------------------------------------- edge and degenerate cases
