@@ -150,13 +150,21 @@ LOT_API size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype)
 
 /*
  * lot_path -- which implementation one lot_attention_fwd_ex call with these parameters takes (host
- * arithmetic only): 0 = the general path (a cost kernel per side, one kernel per Sinkhorn pass, two
- * apply kernels), 1 = the fused tensor-core path (bf16 tensors, d = 64, r <= 64: one persistent
- * kernel for all passes, launched cooperatively, plus a small pivot preparation).  On the fused
- * path with 32 < r <= 64 the first pass keeps the stabilised Gibbs kernel exp(C/eps - rowmax) of
- * the scaling form of Eq. (1)-(2) as bf16 and the later passes iterate on that copy (potentials
- * then agree with an exact float evaluation to about 1e-4, the output to the bf16 rounding of
- * `out`).
+ * arithmetic only):
+ *   0  the general path: a cost kernel per side, one kernel per Sinkhorn pass, two apply kernels.
+ *   1  the streamed tensor-core path (bf16 tensors, d = 64, r <= 64): one persistent kernel for all
+ *      passes, launched cooperatively (it needs as many free SMs as it has thread blocks, at most
+ *      one per SM), plus a small pivot preparation.  With 32 < r <= 64 its first pass keeps the
+ *      stabilised Gibbs kernel exp(C/eps - rowmax) of the scaling form of Eq. (1)-(2) as bf16 in the
+ *      workspace and the later passes stream that copy back.
+ *   2  the resident tensor-core path (same tensors, when a thread block's share of the problem fits
+ *      one SM's tensor memory and shared memory, e.g. B*H*n <= 265216 tokens at r = 64 in long
+ *      sequences, or any number of sequences of up to 1792 tokens): one persistent kernel in which
+ *      that bf16 kernel never leaves the SM between the iterations.  A problem it cannot represent
+ *      (potentials spread over more than 64 binades, a column mass below 2^-80) is recomputed by the
+ *      streamed kernels, which are launched behind it and return at once otherwise.
+ * On paths 1 and 2 the potentials agree with an exact float evaluation to about 1e-4 and the output
+ * to the bf16 rounding of `out`.
  */
 LOT_API int lot_path(int dtype, int B, int H, int n, int d, int r, int iters);
 
@@ -165,6 +173,16 @@ LOT_API int lot_path(int dtype, int B, int H, int n, int d, int r, int iters);
  * parameters launches (host arithmetic only; 0 for iters < 0).
  */
 LOT_API int lot_launch_count(int dtype, int B, int H, int n, int d, int r, int iters);
+
+/*
+ * lot_debug_hook -- switches for the library's own tests; not part of the method.
+ *   what = 1: the thread block `value` of the next resident-path launch never publishes its first
+ *             column partial, so the bounded waits of the blocks that share its slice run out and the
+ *             call ends with LOT_DEV_TIMEOUT (one call only; -1 = none).
+ *   what = 2: limit of every device-side wait of the resident path in nanoseconds (0 = default, 1 s).
+ * Returns LOT_ERR_INVALID_ARG for any other `what`.
+ */
+LOT_API int lot_debug_hook(int what, long long value);
 
 /*
  * lot_attention_fwd_ex -- the whole forward path, Eq. (1)-(4): costs, both solves, apply.

@@ -31,6 +31,7 @@ SIGNATURES = {
     "lot_sinkhorn": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lot_sinkhorn_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _vp]),
     "lot_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
+    "lot_debug_hook": (_i, [_i, ctypes.c_longlong]),
     "lot_path": (_i, [_i, _i, _i, _i, _i, _i, _i]),
     "lot_launch_count": (_i, [_i, _i, _i, _i, _i, _i, _i]),
     "lot_attention_fwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
@@ -146,6 +147,10 @@ def lot_sinkhorn_static(cost, beta, length, eps, iters, g, f=None, plan=None, st
 
 def lot_workspace_bytes(B, H, n, d, r, dtype_code) -> int:
     return lib().lot_workspace_bytes(B, H, n, d, r, dtype_code)
+
+
+def lot_debug_hook(what: int, value: int) -> None:
+    _check(lib().lot_debug_hook(int(what), int(value)), "lot_debug_hook")
 
 
 def lot_path(dtype_code: int, B: int, H: int, n: int, d: int, r: int, iters: int) -> int:

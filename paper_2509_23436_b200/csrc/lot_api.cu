@@ -5,6 +5,7 @@
 
 #include <math.h>
 #include <mutex>
+#include <unordered_map>
 
 namespace {
 
@@ -95,6 +96,30 @@ struct Managed {
 };
 Managed g_managed[kMaxDevices];
 std::mutex g_managed_mu;
+
+// Which path last ran on a workspace, and the tag of that call: the resident path keeps its status word tagged
+// instead of clearing it, so reading it needs the tag (lot_device_status).
+struct WsRecord {
+    int path;
+    unsigned tag;
+    size_t fused_off;
+};
+std::unordered_map<const void *, WsRecord> g_ws_records;
+std::mutex g_ws_mu;
+void remember_ws(const void *ws, int path, unsigned tag, size_t fused_off)
+{
+    std::lock_guard<std::mutex> lock(g_ws_mu);
+    if (g_ws_records.size() > 65536) g_ws_records.clear();
+    g_ws_records[ws] = WsRecord{path, tag, fused_off};
+}
+
+enum { kPathGeneral = 0, kPathStreamed = 1, kPathResident = 2 };
+int choose_path(int dtype, int B, int H, int n, int d, int r)
+{
+    if (!fused_supported(dtype, d, r)) return kPathGeneral;
+    if (B >= 1 && n >= 1 && resident_geometry(dtype, B, H, n, d, r).ok) return kPathResident;
+    return kPathStreamed;
+}
 
 // Scratch of lot_sinkhorn_static: part of the library image, present on every device that loads
 // it.  In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
@@ -219,21 +244,34 @@ size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype)
 {
     if (dtype != LOT_F32 && dtype != LOT_BF16) return 0;
     if (check_dims(B, H, n, r) != LOT_OK || check_d(n, d) != LOT_OK) return 0;
-    if (fused_supported(dtype, d, r)) return fused_layout(B, H, n, d, r).total;
+    const int path = choose_path(dtype, B, H, n, d, r);
+    if (path == kPathResident) return up256(resident_layout(B, H, n, d, r).total) + fused_layout(B, H, n, d, r).total;
+    if (path == kPathStreamed) return fused_layout(B, H, n, d, r).total;
     return attn_layout(B, H, n, d, r, dtype).total;
 }
 
 int lot_path(int dtype, int B, int H, int n, int d, int r, int iters)
 {
-    (void)B; (void)H; (void)n; (void)iters;
-    return fused_supported(dtype, d, r) ? 1 : 0;
+    (void)iters;
+    if (dtype != LOT_F32 && dtype != LOT_BF16) return 0;
+    if (check_dims(B, H, n, r) != LOT_OK || check_d(n, d) != LOT_OK) return 0;
+    return choose_path(dtype, B, H, n, d, r);
 }
 
 int lot_launch_count(int dtype, int B, int H, int n, int d, int r, int iters)
 {
     if (iters < 0) return 0;
-    if (lot_path(dtype, B, H, n, d, r, iters) != 0) return fused_launches(iters);
+    const int path = lot_path(dtype, B, H, n, d, r, iters);
+    if (path == kPathResident) return 1 + fused_launches(iters);    // the two streamed kernels return at once unless asked to redo
+    if (path == kPathStreamed) return fused_launches(iters);
     return 2 + iters + 1 + 2;
+}
+
+int lot_debug_hook(int what, long long value)
+{
+    if (what != 1 && what != 2) return LOT_ERR_INVALID_ARG;
+    resident_debug(what, value);
+    return LOT_OK;
 }
 
 int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
@@ -254,13 +292,30 @@ int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
         !aligned16(out) || !aligned16(g1_out) || !aligned16(g2_out) ||
         (key_len && (reinterpret_cast<uintptr_t>(key_len) & 3u)))
         return LOT_ERR_INVALID_ARG;
-    if (fused_supported(dtype, d, r)) {
-        const size_t need = fused_layout(B, H, n, d, r).total;
+    const int path = choose_path(dtype, B, H, n, d, r);
+    if (path != kPathGeneral) {
+        const size_t res_bytes = path == kPathResident ? up256(resident_layout(B, H, n, d, r).total) : 0;
+        const size_t need = res_bytes + fused_layout(B, H, n, d, r).total;
         if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < need) return LOT_ERR_WORKSPACE;
+        cudaStream_t s = (cudaStream_t)stream;
+        unsigned tag = 0;
+        const unsigned *redo = nullptr;
+        if (path == kPathResident) {
+            if (resident_attention(q, k, v, z, beta, key_len, B, H, n, d, r, eps, iters, out, g1_out, g2_out, ws, &tag, s) !=
+                cudaSuccess) {
+                (void)cudaGetLastError();
+                return LOT_ERR_CUDA;
+            }
+            redo = at<unsigned>(ws, resident_layout(B, H, n, d, r).status + 8);
+        }
+        remember_ws(ws, path, tag, res_bytes);
+        // behind a resident launch the streamed kernels run only if that launch asked for it (a problem outside the
+        // range of the stored bf16 kernel); alone they are the path
         cudaError_t e = fused_attention(q, k, v, z, beta, key_len, B, H, n, d, r, eps, iters, out, g1_out, g2_out,
-                                        ws, (cudaStream_t)stream);
+                                        at<char>(ws, res_bytes), redo, tag, s);
         return e == cudaSuccess ? LOT_OK : LOT_ERR_CUDA;
     }
+    remember_ws(ws, kPathGeneral, 0, 0);
     AttnLayout A = attn_layout(B, H, n, d, r, dtype);
     const bool wide = dtype == LOT_F32;
     const size_t lt = wide ? 8 : 4;
@@ -347,8 +402,28 @@ int lot_device_status(const void *ws, lot_stream_t stream, int *status)
         if (!ws) { *status = 0; return LOT_OK; }
     }
     cudaStream_t s = (cudaStream_t)stream;
-    if (cudaMemcpyAsync(status, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOT_ERR_CUDA;
+    WsRecord rec{kPathGeneral, 0, 0};
+    {
+        std::lock_guard<std::mutex> lock(g_ws_mu);
+        auto it = g_ws_records.find(ws);
+        if (it != g_ws_records.end()) rec = it->second;
+    }
+    if (rec.path != kPathResident) {
+        if (cudaMemcpyAsync(status, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOT_ERR_CUDA;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return LOT_ERR_CUDA;
+        return LOT_OK;
+    }
+    // resident path: {flags | tag << 32, redo word} at the start, the streamed kernels' word behind the resident block
+    unsigned head[4] = {0, 0, 0, 0};
+    int streamed = 0;
+    if (cudaMemcpyAsync(head, ws, sizeof(head), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (cudaMemcpyAsync(&streamed, static_cast<const char *>(ws) + rec.fused_off, sizeof(int), cudaMemcpyDeviceToHost, s) !=
+        cudaSuccess)
+        return LOT_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return LOT_ERR_CUDA;
+    const int mine = head[1] == rec.tag ? (int)head[0] : 0;
+    // a call that was recomputed reports the recomputation's flags (and a timeout of the first attempt, if any)
+    *status = head[2] == rec.tag ? (streamed | (mine & LOT_DEV_TIMEOUT)) : (mine | streamed);
     return LOT_OK;
 }
 

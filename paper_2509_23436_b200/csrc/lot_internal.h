@@ -69,9 +69,27 @@ struct FusedLayout {
 bool fused_supported(int dtype, int d, int r);
 void fused_geometry(int B, int H, int n, int *q, int *ctas, int *maxslots, int *cps);
 FusedLayout fused_layout(int B, int H, int n, int d, int r);
+// redo != nullptr: both kernels return at once unless *redo == redo_tag (the call behind a resident launch)
 cudaError_t fused_attention(const void *q, const void *k, const void *v, const float *z, const float *beta,
                             const int32_t *key_len, int B, int H, int n, int d, int r, float eps, int iters,
-                            void *out, float *g1_out, float *g2_out, void *ws, cudaStream_t st);
+                            void *out, float *g1_out, float *g2_out, void *ws, const unsigned *redo, unsigned redo_tag,
+                            cudaStream_t st);
 int fused_launches(int iters);
+
+// ---- resident tensor-core path (lot_resident.cu): bf16 tensors, d = 64, r <= 64, tiles fit one SM's TMEM + shared memory ----
+struct ResidentGeom {
+    bool ok;
+    int ctas, whole, wave_slices, maxslots, TPS, NT;
+};
+struct ResidentLayout {
+    size_t status, part, wflag, wpart, spill, total;
+};
+int device_sm_count();                       // SM count of the current device (cached per device)
+ResidentGeom resident_geometry(int dtype, int B, int H, int n, int d, int r);
+ResidentLayout resident_layout(int B, int H, int n, int d, int r);
+cudaError_t resident_attention(const void *q, const void *k, const void *v, const float *z, const float *beta,
+                               const int32_t *key_len, int B, int H, int n, int d, int r, float eps, int iters,
+                               void *out, float *g1_out, float *g2_out, void *ws, unsigned *tag_out, cudaStream_t st);
+void resident_debug(int what, long long value);   // test hooks: 1 = block that skips its first publish (one call), 2 = wait limit in ns
 
 } // namespace lot

@@ -49,7 +49,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait.  `abort_flag` lives in shared memory; `status` is the global status word.  The common case
 // (phase already complete, or complete within the first suspended try) stays inline; the timed loop does not.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
     uint64_t t0 = 0;
     for (uint32_t it = 0;; ++it) {
