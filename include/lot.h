@@ -76,7 +76,9 @@ enum lot_dtype { LOT_F32 = 0, LOT_BF16 = 1 };
 enum lot_device_flag {
     LOT_DEV_NONFINITE = 1, /* a pivot potential became inf/nan (e.g. beta_t <= 0) */
     LOT_DEV_EMPTY = 2,     /* a key_len entry was <= 0: that slice has no key mass; its output is zeros */
-    LOT_DEV_TIMEOUT = 4    /* a bounded device-side wait gave up; results of the call are invalid */
+    LOT_DEV_TIMEOUT = 4,   /* a bounded device-side wait gave up; results of the call are invalid */
+    LOT_DEV_RECOMPUTED = 8 /* information only: the resident path could not represent the problem (see lot_path)
+                              and the streamed kernels recomputed the call; the results are valid */
 };
 
 /* Library version: major*10000 + minor*100 + patch. */
@@ -157,12 +159,13 @@ LOT_API size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype)
  *      one per SM), plus a small pivot preparation.  With 32 < r <= 64 its first pass keeps the
  *      stabilised Gibbs kernel exp(C/eps - rowmax) of the scaling form of Eq. (1)-(2) as bf16 in the
  *      workspace and the later passes stream that copy back.
- *   2  the resident tensor-core path (same tensors, when a thread block's share of the problem fits
- *      one SM's tensor memory and shared memory, e.g. B*H*n <= 265216 tokens at r = 64 in long
- *      sequences, or any number of sequences of up to 1792 tokens): one persistent kernel in which
- *      that bf16 kernel never leaves the SM between the iterations.  A problem it cannot represent
- *      (potentials spread over more than 64 binades, a column mass below 2^-80) is recomputed by the
- *      streamed kernels, which are launched behind it and return at once otherwise.
+ *   2  the resident tensor-core path (same tensors; taken for r <= 32 when every thread block can
+ *      hold whole sequences, up to 1792 tokens, and all of its share at once): one persistent kernel in
+ *      which that bf16 kernel never leaves the SM (tensor memory and shared memory) between the
+ *      iterations.  A problem it cannot represent (potentials spread over more than 96 binades, a
+ *      column mass below 2^-80) is recomputed by the streamed kernels, which are launched behind it
+ *      and return at once otherwise (device flag LOT_DEV_RECOMPUTED).  It can run many more shapes
+ *      (lot_debug_hook what = 4), but measured no faster there.
  * On paths 1 and 2 the potentials agree with an exact float evaluation to about 1e-4 and the output
  * to the bf16 rounding of `out`.
  */
@@ -180,6 +183,11 @@ LOT_API int lot_launch_count(int dtype, int B, int H, int n, int d, int r, int i
  *             column partial, so the bounded waits of the blocks that share its slice run out and the
  *             call ends with LOT_DEV_TIMEOUT (one call only; -1 = none).
  *   what = 2: limit of every device-side wait of the resident path in nanoseconds (0 = default, 1 s).
+ *   what = 3: device address of a trace buffer (8002 64-bit words, zeroed by the caller) into which thread block 0 of
+ *             the resident path logs (event code, global timer) pairs, or 0 to stop; for profiling.
+ *   what = 4: 1 or 2 makes lot_attention_fwd_ex take tensor-core path 1 or 2 of lot_path wherever that path can run
+ *             at all (the default choice is by measured speed); -1 restores the default.  lot_path and
+ *             lot_workspace_bytes follow the switch.
  * Returns LOT_ERR_INVALID_ARG for any other `what`.
  */
 LOT_API int lot_debug_hook(int what, long long value);

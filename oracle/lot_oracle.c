@@ -77,15 +77,29 @@ static double lse(const double *a, const unsigned char *skip, int len, int strid
  *      Tokens with m_i == 0 take no part (f_i = -inf, P_i: = 0).
  *
  *      g [r], f [n], P [n,r] are outputs; f and P may be NULL. */
+void lot_oracle_sinkhorn_from(const double *C, const double *beta, const double *m,
+                              int n, int r, double eps, int iters, const double *g0,
+                              double *g, double *f, double *P);
+
 void lot_oracle_sinkhorn(const double *C, const double *beta, const double *m,
                          int n, int r, double eps, int iters,
                          double *g, double *f, double *P)
+{
+    lot_oracle_sinkhorn_from(C, beta, m, n, r, eps, iters, NULL, g, f, P);
+}
+
+/* The same iteration started from a given pivot potential g0 (NULL = zeros): the state of the
+ * iteration between two passes is g alone, so T1 iterations followed by T2 more from the
+ * exported g are T1 + T2 iterations (warm start across layers or steps). */
+void lot_oracle_sinkhorn_from(const double *C, const double *beta, const double *m,
+                              int n, int r, double eps, int iters, const double *g0,
+                              double *g, double *f, double *P)
 {
     double *fl = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
     double *tmp = (double *)malloc(sizeof(double) * (size_t)((n > r ? n : r) + 1));
     unsigned char *dead = (unsigned char *)malloc((size_t)(n > 0 ? n : 1));
     for (int i = 0; i < n; ++i) dead[i] = !(m[i] > 0.0);
-    for (int t = 0; t < r; ++t) g[t] = 0.0;
+    for (int t = 0; t < r; ++t) g[t] = g0 ? g0[t] : 0.0;
 
     for (int it = 0; it <= iters; ++it) {
         /* token-side update with the current g */
@@ -178,6 +192,63 @@ void lot_oracle_head(const double *q, const double *k, const double *v,
     if (P1o) memcpy(P1o, P1, sizeof(double) * nr);
     if (P2o) memcpy(P2o, P2, sizeof(double) * nr);
     free(C1); free(C2); free(P1); free(P2); free(ga); free(gb);
+}
+
+/* ---- One head with its own query and key counts (cross-attention: Appendix "Bidirectional scope",
+ *      closing paragraph), arbitrary marginals a [nq], b [nk] (Section "Empirical measures and
+ *      pivot": weights p^1, p^2 on the simplex; zero weight removes the token) and optional
+ *      starting potentials g1_0, g2_0 [r] (NULL = zeros).  v, out have dv columns. */
+void lot_oracle_head_x(const double *q, const double *k, const double *v,
+                       const double *z, const double *beta,
+                       const double *a, const double *b,
+                       int nq, int nk, int d, int dv, int r, double eps, int iters,
+                       const double *g1_0, const double *g2_0,
+                       double *out, double *g1, double *g2, double *P1o, double *P2o)
+{
+    size_t n1 = (size_t)nq * r, n2 = (size_t)nk * r;
+    double *C1 = (double *)malloc(sizeof(double) * (n1 ? n1 : 1));
+    double *C2 = (double *)malloc(sizeof(double) * (n2 ? n2 : 1));
+    double *P1 = (double *)malloc(sizeof(double) * (n1 ? n1 : 1));
+    double *P2 = (double *)malloc(sizeof(double) * (n2 ? n2 : 1));
+    double *ga = (double *)malloc(sizeof(double) * (size_t)r);
+    double *gb = (double *)malloc(sizeof(double) * (size_t)r);
+    lot_oracle_cost(q, z, nq, d, r, C1);
+    lot_oracle_cost(k, z, nk, d, r, C2);
+    lot_oracle_sinkhorn_from(C1, beta, a, nq, r, eps, iters, g1_0, ga, NULL, P1);
+    lot_oracle_sinkhorn_from(C2, beta, b, nk, r, eps, iters, g2_0, gb, NULL, P2);
+    lot_oracle_apply(P1, P2, beta, a, v, nq, nk, r, dv, out);
+    if (g1) memcpy(g1, ga, sizeof(double) * (size_t)r);
+    if (g2) memcpy(g2, gb, sizeof(double) * (size_t)r);
+    if (P1o) memcpy(P1o, P1, sizeof(double) * n1);
+    if (P2o) memcpy(P2o, P2, sizeof(double) * n2);
+    free(C1); free(C2); free(P1); free(P2); free(ga); free(gb);
+}
+
+/* ---- Eq. (5): the [CLS] row keeps a plain softmax over the keys,
+ *      alpha_j = exp(tau <q_cls, k_j>) / sum_l exp(tau <q_cls, k_l>),  out_cls = sum_j alpha_j v_j
+ *      (tau is the paper's beta > 0 of Eq. (5), renamed because beta names the pivot masses here).
+ *      Keys with alive[j] == 0 are left out (alive == NULL: all keys). */
+void lot_oracle_cls_row(const double *q0, const double *k, const double *v, const unsigned char *alive,
+                        int nk, int d, int dv, double tau, double *out0)
+{
+    double *s = (double *)malloc(sizeof(double) * (size_t)(nk > 0 ? nk : 1));
+    double mx = -INFINITY;
+    for (int j = 0; j < nk; ++j) {
+        double acc = 0.0;
+        for (int c = 0; c < d; ++c) acc += q0[c] * k[(size_t)j * d + c];
+        s[j] = tau * acc;
+        if ((!alive || alive[j]) && s[j] > mx) mx = s[j];
+    }
+    double den = 0.0;
+    for (int j = 0; j < nk; ++j)
+        if (!alive || alive[j]) den += exp(s[j] - mx);
+    for (int c = 0; c < dv; ++c) {
+        double acc = 0.0;
+        for (int j = 0; j < nk; ++j)
+            if (!alive || alive[j]) acc += exp(s[j] - mx) / den * v[(size_t)j * dv + c];
+        out0[c] = acc;
+    }
+    free(s);
 }
 
 /* ---- All (batch, head) slices.  q,k,v,out [B,H,n,d]; z [H,r,d]; beta [H,r]

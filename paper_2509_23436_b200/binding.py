@@ -15,7 +15,7 @@ import torch
 
 LOT_F32, LOT_BF16 = 0, 1
 LOT_OK = 0
-LOT_DEV_NONFINITE, LOT_DEV_EMPTY, LOT_DEV_TIMEOUT = 1, 2, 4
+LOT_DEV_NONFINITE, LOT_DEV_EMPTY, LOT_DEV_TIMEOUT, LOT_DEV_RECOMPUTED = 1, 2, 4, 8
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblot.so")
 _lib = None

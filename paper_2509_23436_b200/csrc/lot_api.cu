@@ -4,6 +4,7 @@
 #include "lot_internal.h"
 
 #include <math.h>
+#include <atomic>
 #include <mutex>
 #include <unordered_map>
 
@@ -114,10 +115,21 @@ void remember_ws(const void *ws, int path, unsigned tag, size_t fused_off)
 }
 
 enum { kPathGeneral = 0, kPathStreamed = 1, kPathResident = 2 };
+std::atomic<int> g_force_path{-1};      // test hook: 1 or 2 picks that tensor-core path wherever it can run
 int choose_path(int dtype, int B, int H, int n, int d, int r)
 {
     if (!fused_supported(dtype, d, r)) return kPathGeneral;
-    if (B >= 1 && n >= 1 && resident_geometry(dtype, B, H, n, d, r).ok) return kPathResident;
+    const bool res_ok = B >= 1 && n >= 1 && resident_geometry(dtype, B, H, n, d, r).ok;
+    const int force = g_force_path.load();
+    if (force == kPathStreamed) return kPathStreamed;
+    if (force == kPathResident) return res_ok ? kPathResident : kPathStreamed;
+    // Measured on B200 (see the design notes): the resident kernel wins where the streamed one has no stored-kernel
+    // passes (r <= 32, every pass recomputes logits and exponentials) and every thread block holds its whole share at
+    // once (whole slices, one wave); elsewhere the streamed kernel is as fast or faster.
+    if (res_ok && r <= 32) {
+        const ResidentGeom G = resident_geometry(dtype, B, H, n, d, r);
+        if (G.whole && (long long)B * H <= (long long)G.ctas * G.wave_slices) return kPathResident;
+    }
     return kPathStreamed;
 }
 
@@ -269,8 +281,9 @@ int lot_launch_count(int dtype, int B, int H, int n, int d, int r, int iters)
 
 int lot_debug_hook(int what, long long value)
 {
-    if (what != 1 && what != 2) return LOT_ERR_INVALID_ARG;
-    resident_debug(what, value);
+    if (what < 1 || what > 4) return LOT_ERR_INVALID_ARG;
+    if (what == 4) g_force_path.store((int)value);
+    else resident_debug(what, value);
     return LOT_OK;
 }
 
@@ -423,7 +436,7 @@ int lot_device_status(const void *ws, lot_stream_t stream, int *status)
     if (cudaStreamSynchronize(s) != cudaSuccess) return LOT_ERR_CUDA;
     const int mine = head[1] == rec.tag ? (int)head[0] : 0;
     // a call that was recomputed reports the recomputation's flags (and a timeout of the first attempt, if any)
-    *status = head[2] == rec.tag ? (streamed | (mine & LOT_DEV_TIMEOUT)) : (mine | streamed);
+    *status = head[2] == rec.tag ? (LOT_DEV_RECOMPUTED | streamed | (mine & LOT_DEV_TIMEOUT)) : (mine | streamed);
     return LOT_OK;
 }
 

@@ -24,7 +24,7 @@
 // 2 that spill to global memory and come back into the two auxiliary buffers) and 448 TMEM columns of query-side
 // tiles; problems beyond that take the streamed kernel (lot_fused.cu).
 //
-// The stored bf16 kernel cannot represent a problem whose potentials spread over more than 64 binades or whose
+// The stored bf16 kernel cannot represent a problem whose potentials spread over more than 96 binades or whose
 // column mass underflows; such a call raises the redo word and the streamed kernel, launched behind this one on
 // the same stream, recomputes it (it returns at once when the word is not raised).
 //
@@ -59,6 +59,10 @@ constexpr int kThreads = 384;
 constexpr int kWorkers = 256;
 constexpr int kAccCol = 448;                        // 64 TMEM columns of accumulator behind the query-side tiles
 constexpr float kPlainFloor = 8.2718061e-25f;       // 2^-80: smallest column mass the plain sums may report
+// Largest spread of the pivot potentials (in binades) the stored kernel serves: with w_t = 2^(G_t - max G) >= 2^-96 a row
+// sum is at least 2^-96, its reciprocal and the column sums stay far inside the float range, and an entry that matters
+// for a row (within 2^-24 of the row's largest product K~ w) is at least 2^-120, which bf16 still holds.
+constexpr float kMaxSpread = 96.f;
 
 struct alignas(64) ResParams {
     CUtensorMap tmQ, tmK, tmV, tmO;  // [BH][n][64] bf16, box 64 x 128 x 1, 128-byte swizzle
@@ -84,6 +88,7 @@ struct alignas(64) ResParams {
     float eps_ln2;
     unsigned long long wait_ns;      // limit of every device-side wait
     int skip_publish_cta;            // test hook: that block never publishes its first column partial (-1: none)
+    unsigned long long *trace;       // profiling hook: block 0 logs (event, nanoseconds) pairs here, or nullptr
 };
 
 // ---------------------------------------------------------------------------------------
@@ -343,32 +348,43 @@ __device__ __noinline__ void raise_flag(const ResParams &P, unsigned flag)
     }
 }
 
-// Diagnostic record of a wait that gave up: (tag << 32) | block << 20 | phase << 16 | barrier << 8 | warp, one word per
-// warp behind the status and redo words (barrier >= 100: a poll of global memory).
-__device__ __noinline__ void record_timeout(const Ctx &c, int barid)
+// Profiling hook: block 0 appends (warp << 32 | code, global timer) to the trace buffer (word 0 counts the entries, at
+// most 4000).
+__device__ __forceinline__ void trace(const Ctx &c, unsigned code)
 {
-    unsigned long long *info = c.P.status + 2 + blockIdx.x * 12 + c.warp;
-    const unsigned long long mine = ((unsigned long long)c.P.tag << 32) | ((unsigned)blockIdx.x << 20) |
-                                    ((unsigned)(c.M->phase & 15) << 16) | ((unsigned)(barid & 255) << 8) | (unsigned)c.warp;
-    const unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(info);
-    if ((unsigned)(old >> 32) != c.P.tag) atomicCAS(info, old, mine);
+    if (c.P.trace != nullptr && blockIdx.x == 0 && c.lane == 0) {
+        const unsigned long long n = atomicAdd(c.P.trace, 1ull);
+        if (n < 4000) { c.P.trace[1 + 2 * n] = ((unsigned long long)c.warp << 32) | code; c.P.trace[2 + 2 * n] = global_timer_ns(); }
+    }
 }
 
-__device__ __noinline__ bool bar_wait_slow(const Ctx &c, uint32_t b, uint32_t parity)
+// Diagnostic record of a wait that gave up: (tag << 32) | block << 20 | phase << 16 | barrier << 8 | warp, one word per
+// warp behind the status and redo words (barrier >= 100: a poll of global memory).
+__device__ __noinline__ void record_timeout(const ResParams *P, volatile Misc *M, int warp, int barid)
+{
+    unsigned long long *info = P->status + 2 + blockIdx.x * 12 + warp;
+    const unsigned long long mine = ((unsigned long long)P->tag << 32) | ((unsigned)blockIdx.x << 20) |
+                                    ((unsigned)(M->phase & 15) << 16) | ((unsigned)(barid & 255) << 8) | (unsigned)warp;
+    const unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(info);
+    if ((unsigned)(old >> 32) != P->tag) atomicCAS(info, old, mine);
+}
+
+// The timed part of a barrier wait; the cold path takes plain values so that the callers' context stays in registers.
+__device__ __noinline__ bool bar_wait_slow(uint32_t b, uint32_t parity, uint32_t bar0, volatile Misc *M, const ResParams *P, int warp)
 {
     uint64_t t0 = 0;
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(b, parity)) return true;
         if ((it & 63u) == 63u) {
-            if (c.M->abort) return false;
+            if (M->abort) return false;
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > c.P.wait_ns) break;
+            else if (now - t0 > P->wait_ns) break;
         }
     }
-    c.M->abort = 1;
-    record_timeout(c, (int)((b - c.bar(0)) >> 3));
-    raise_flag(c.P, 4 /* LOT_DEV_TIMEOUT */);
+    M->abort = 1;
+    record_timeout(P, M, warp, (int)((b - bar0) >> 3));
+    raise_flag(*P, 4 /* LOT_DEV_TIMEOUT */);
     return false;
 }
 __device__ __forceinline__ bool bar_wait(const Ctx &c, int id, uint32_t parity)
@@ -376,7 +392,7 @@ __device__ __forceinline__ bool bar_wait(const Ctx &c, int id, uint32_t parity)
     const uint32_t b = c.bar(id);
     if (mbar_try_wait(b, parity)) return true;
     if (mbar_try_wait(b, parity)) return true;
-    return bar_wait_slow(c, b, parity);
+    return bar_wait_slow(b, parity, c.bar(0), c.M, &c.P, c.warp);
 }
 // whole-warp wait with a warp-uniform verdict
 __device__ __forceinline__ bool warp_wait(const Ctx &c, int id, uint32_t parity)
@@ -517,7 +533,7 @@ __device__ __forceinline__ void tma_tile(const Ctx &c, const CUtensorMap *map, i
     tma_load_3d(c.bufa(b), map, c.bar(barid), 0, row, outer);
 }
 
-__device__ __noinline__ void producer_x(const Ctx &c)
+__device__ __noinline__ void producer_x(const Ctx c)
 {
     const ResParams &P = c.P;
     const Misc *M = c.M;
@@ -544,13 +560,21 @@ __device__ __noinline__ void producer_x(const Ctx &c)
             if (!bar_wait(c, bEmpty + b, f & 1)) return;
     }
 }
-__device__ __noinline__ void producer_s(const Ctx &c)
+__device__ __noinline__ void producer_s(const Ctx c)
 {
-    const int nSp = max(c.M->nK - kSlots, 0);
-    if (c.P.T < 2) return;
-    for (int o = 0; o < nSp; ++o) tma_tile(c, &c.P.tmS, kSlots + o, bSFull + o, 0, blockIdx.x * 2 + o);
+    const Misc *M = c.M;
+    const int nSp = max(M->nK - kSlots, 0);
+    if (c.P.T >= 2)
+        for (int o = 0; o < nSp; ++o) tma_tile(c, &c.P.tmS, kSlots + o, bSFull + o, 0, blockIdx.x * 2 + o);
+    // the value tiles of phase W: asked into the L2 now, while the Sinkhorn passes need no memory traffic
+    for (int k = 0; k < M->nK; ++k) {
+        int seg, t;
+        locate(M, 1, k, seg, t);
+        asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                     ::"l"(reinterpret_cast<uint64_t>(&c.P.tmV)), "r"(0), "r"(t * kTileRows), "r"(M->seg[seg].s) : "memory");
+    }
 }
-__device__ __noinline__ void producer_w(const Ctx &c)
+__device__ __noinline__ void producer_w(const Ctx c)
 {
     const ResParams &P = c.P;
     const Misc *M = c.M;
@@ -577,7 +601,7 @@ __device__ __noinline__ void producer_w(const Ctx &c)
 __device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; }
 
 template <int RP>
-__device__ __noinline__ void mma_x(const Ctx &c)
+__device__ __noinline__ void mma_x(const Ctx c)
 {
     const Misc *M = c.M;
     const int nX = M->nQ + M->nK, nRing = M->nQ + max(M->nK - kSlots, 0);
@@ -595,6 +619,7 @@ __device__ __noinline__ void mma_x(const Ctx &c)
         if (ok && k >= 1) ok = warp_wait(c, bAccEmpty + ((k - 1) & 1), ((k - 1) >> 1) & 1);
         if (!ok) break;
         tc_fence_after();
+        trace(c, 0x100 + k);
         int seg, t;
         const int side = k < M->nQ ? 0 : 1;
         locate(M, side, side ? k - M->nQ : k, seg, t);
@@ -619,7 +644,7 @@ __device__ __noinline__ void mma_x(const Ctx &c)
 // product would cost the output three times its own bf16 rounding).  Both parts pass through the tile's one buffer:
 // the hi-part MMAs of position k, the hi-part MMAs of position k + 1 (the other quad's), then the lo-part MMAs of
 // position k, which its quad has written over the hi part meanwhile.
-__device__ __noinline__ void mma_w(const Ctx &c)
+__device__ __noinline__ void mma_w(const Ctx c)
 {
     const Misc *M = c.M;
     const int nSp = max(M->nK - kSlots, 0);
@@ -666,7 +691,7 @@ __device__ __noinline__ void mma_w(const Ctx &c)
 }
 
 template <int RP>
-__device__ __noinline__ void mma_o(const Ctx &c)
+__device__ __noinline__ void mma_o(const Ctx c)
 {
     const Misc *M = c.M;
     const uint32_t tm = c.M->tmem + kAccCol;
@@ -710,7 +735,7 @@ __device__ __forceinline__ unsigned long long *part_slot(const ResParams &P, int
 }
 
 template <int RP>
-__device__ __noinline__ void publisher(const Ctx &c, int p_lo, int p_hi)
+__device__ __noinline__ void publisher(const Ctx c, int p_lo, int p_hi)
 {
     const ResParams &P = c.P;
     const Misc *M = c.M;
@@ -725,6 +750,7 @@ __device__ __noinline__ void publisher(const Ctx &c, int p_lo, int p_hi)
             const SegInfo &g = M->seg[sg];
             if (ok) ok = warp_wait(c, bP2, nph & 1);
             ++nph;
+            trace(c, 0x600 + p * 4 + sg);
             // column masses of this block's tiles: the four lane quarters' rows, times the weights of this pass
             float a0 = 0.f, a1 = 0.f;
             if (mine && ok) {
@@ -753,7 +779,7 @@ struct GatherState {
 };
 
 template <int RP>
-__device__ __noinline__ void gatherer(const Ctx &c, GatherState &st, int p_lo, int p_hi)
+__device__ __noinline__ void gatherer(const Ctx c, GatherState &st, int p_lo, int p_hi)
 {
     const ResParams &P = c.P;
     const Misc *M = c.M;
@@ -779,17 +805,18 @@ __device__ __noinline__ void gatherer(const Ctx &c, GatherState &st, int p_lo, i
                 // all slots of the (slice, side), polled until their tags match, summed in slot order
                 const unsigned tag = P.tag + (unsigned)p + 1u;
                 const unsigned long long *src = part_slot(P, RP, p, sg & 1, g.s, 0) + c0;
-                for (int p0 = 0; p0 < g.nslots && ok; p0 += 4) {
-                    unsigned long long w[4][2];
+                constexpr int kBatch = 12;          // slots polled together: their loads are all in flight at once
+                for (int p0 = 0; p0 < g.nslots && ok; p0 += kBatch) {
+                    unsigned long long w[kBatch][2];
                     uint64_t t0 = 0;
                     for (uint32_t tries = 0;; ++tries) {
                         bool ready = true;
                         if (mine) {
 #pragma unroll
-                            for (int u = 0; u < 4; ++u)
+                            for (int u = 0; u < kBatch; ++u)
                                 if (p0 + u < g.nslots) ld_tagged2(src + (size_t)(p0 + u) * RP, w[u][0], w[u][1]);
 #pragma unroll
-                            for (int u = 0; u < 4; ++u)
+                            for (int u = 0; u < kBatch; ++u)
                                 if (p0 + u < g.nslots)
                                     ready = ready && (unsigned)(w[u][0] >> 32) == tag && (unsigned)(w[u][1] >> 32) == tag;
                         }
@@ -801,7 +828,7 @@ __device__ __noinline__ void gatherer(const Ctx &c, GatherState &st, int p_lo, i
                             else if (now - t0 > P.wait_ns) giveup = true;
                         }
                         if (__any_sync(0xffffffffu, giveup)) {
-                            if (c.lane == 0) { c.M->abort = 1; record_timeout(c, 100 + sg); raise_flag(P, 4 /* LOT_DEV_TIMEOUT */); }
+                            if (c.lane == 0) { c.M->abort = 1; record_timeout(&P, c.M, c.warp, 100 + sg); raise_flag(P, 4 /* LOT_DEV_TIMEOUT */); }
                             ok = false;
                             break;
                         }
@@ -809,7 +836,7 @@ __device__ __noinline__ void gatherer(const Ctx &c, GatherState &st, int p_lo, i
                     }
                     if (!ok || !mine) continue;
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
+                    for (int u = 0; u < kBatch; ++u)
                         if (p0 + u < g.nslots) { s0 += __uint_as_float((unsigned)w[u][0]); s1 += __uint_as_float((unsigned)w[u][1]); }
                 }
                 if (!ok) continue;
@@ -841,8 +868,8 @@ __device__ __noinline__ void gatherer(const Ctx &c, GatherState &st, int p_lo, i
                 gmn = fminf(gmn, __shfl_xor_sync(0xffffffffu, gmn, off));
             }
             // what the stored bf16 kernel cannot carry: a column mass outside the plain range, potentials spread over
-            // more than 64 binades (they decide how small a row sum can get).  NaN fails the comparison too.
-            if (__any_sync(0xffffffffu, bad) || !(gmx - gmn <= 64.f)) {
+            // more than kMaxSpread binades.  NaN fails the comparison too.
+            if (__any_sync(0xffffffffu, bad) || !(gmx - gmn <= kMaxSpread)) {
                 if (c.lane == 0) *reinterpret_cast<volatile unsigned *>(P.redo) = P.tag;
             }
             if (mine) {
@@ -852,6 +879,7 @@ __device__ __noinline__ void gatherer(const Ctx &c, GatherState &st, int p_lo, i
                 *reinterpret_cast<float2 *>(c.sW + sg * 64 + c0) = w;
             }
             warp_arrive(c, bWReady + sg);
+            trace(c, 0x700 + p * 4 + sg);
         }
 }
 
@@ -884,7 +912,7 @@ __device__ __forceinline__ bool flush_partial(const Ctx &c, const WorkerId &id, 
 
 // ---- phase X: pivots -> MMA operands; logits -> stabilised kernel tiles and the first column sums
 template <int RP>
-__device__ __noinline__ void worker_x(const Ctx &c, const WorkerId &id)
+__device__ __noinline__ void worker_x(const Ctx c, const WorkerId id)
 {
     constexpr int X = RP / 8;            // repeats of the 8-column pattern of the accumulator load
     const ResParams &P = c.P;
@@ -940,15 +968,18 @@ __device__ __noinline__ void worker_x(const Ctx &c, const WorkerId &id)
             ++ntile;
             if (!ok) continue;
             tc_fence_after();
+            trace(c, 0x200 + k);
+            // both 16-lane halves into registers, then the accumulator goes back to the MMA issuer at once
+            float vv[2][4 * X];
+            tmem_ld_acc<X>(id.lane_addr + kAccCol, vv[0]);
+            tmem_ld_acc<X>(id.lane_addr + (16u << 16) + kAccCol, vv[1]);
+            tmem_wait_ld();
+            tc_fence_before();
+            warp_arrive(c, bAccEmpty + id.quad);
+            trace(c, 0x300 + k);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                float v[4 * X];
-                tmem_ld_acc<X>(id.lane_addr + ((uint32_t)(half * 16) << 16) + kAccCol, v);
-                tmem_wait_ld();
-                if (half == 1) {
-                    tc_fence_before();
-                    warp_arrive(c, bAccEmpty + id.quad);
-                }
+                float (&v)[4 * X] = vv[half];
                 const int rinA = id.w4 * 32 + half * 16 + id.rq;          // row inside the tile; row B = row A + 8
                 const int rowA = t * kTileRows + rinA, rowB = rowA + 8;
                 if (P.r < RP) {
@@ -1080,13 +1111,13 @@ __device__ __forceinline__ int word_col(const WorkerId &id, int e)
 }
 // row sums s_j = sum_t K~_jt w_t of the thread's four rows (complete after the two quad shuffles)
 template <int NW>
-__device__ __forceinline__ void row_sums(const uint32_t (&d)[4][NW], const float2 (&w2)[NW], float2 (&kf)[4][NW], float (&sr)[4])
+__device__ __forceinline__ void row_sums(const uint32_t (&d)[4][NW], const float2 (&w2)[NW], float (&sr)[4])
 {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         float2 sa = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int e = 0; e < NW; ++e) { kf[j][e] = unpack_bf16(d[j][e]); sa = __ffma2_rn(kf[j][e], w2[e], sa); }
+        for (int e = 0; e < NW; ++e) sa = __ffma2_rn(unpack_bf16(d[j][e]), w2[e], sa);
         sr[j] = sa.x + sa.y;
     }
 #pragma unroll
@@ -1118,16 +1149,16 @@ __device__ __forceinline__ bool pass_segment(const Ctx &c, const WorkerId &id, i
             if (idx < nSp && ok) ok = warp_wait(c, bSFull + idx, 0);
             load_rows<RP, false>(c, id, 0, c.buf(idx < nSp ? kSlots + idx : idx - nSp), d);
         }
-        float2 kf[4][NW];
         float sr[4];
-        row_sums<NW>(d, w2, kf, sr);
+        row_sums<NW>(d, w2, sr);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int row = t * kTileRows + id.w4 * 32 + j * 8 + id.rq;
             const float u = row < g.nvalid ? __fdividef(1.f, sr[j]) : 0.f;
             const float2 uu = make_float2(u, u);
+            // unpacked a second time on purpose: the float pairs of a whole tile would not fit the registers
 #pragma unroll
-            for (int e = 0; e < NW; ++e) c2[e] = __ffma2_rn(kf[j][e], uu, c2[e]);
+            for (int e = 0; e < NW; ++e) c2[e] = __ffma2_rn(unpack_bf16(d[j][e]), uu, c2[e]);
         }
     }
     float a[2 * NW];
@@ -1139,7 +1170,7 @@ __device__ __forceinline__ bool pass_segment(const Ctx &c, const WorkerId &id, i
 }
 
 template <int RP>
-__device__ __noinline__ void worker_s(const Ctx &c, const WorkerId &id)
+__device__ __noinline__ void worker_s(const Ctx c, const WorkerId id)
 {
     const Misc *M = c.M;
     int nflush = 0;
@@ -1149,7 +1180,9 @@ __device__ __noinline__ void worker_s(const Ctx &c, const WorkerId &id)
             const int sg = seg_at(i);
             if (!seg_active(M, sg)) continue;
             // weights of this pass: the gather of pass p - 1 (pass 0's finished before this phase began)
+            trace(c, 0x400 + p * 4 + sg);
             if (p >= 2 && ok) ok = warp_wait(c, bWReady + sg, p & 1);
+            trace(c, 0x500 + p * 4 + sg);
             if (sg & 1) ok = pass_segment<RP, false>(c, id, sg, nflush, ok);
             else ok = pass_segment<RP, true>(c, id, sg, nflush, ok);
         }
@@ -1157,7 +1190,7 @@ __device__ __noinline__ void worker_s(const Ctx &c, const WorkerId &id)
 
 // ---- phase W: closing token update of the key side, value rows scaled by 1/s_j, W = K~2^T V' on tensor cores
 template <int RP>
-__device__ __noinline__ void worker_w(const Ctx &c, const WorkerId &id)
+__device__ __noinline__ void worker_w(const Ctx c, const WorkerId id)
 {
     constexpr int NW = RP / 8;
     const ResParams &P = c.P;
@@ -1180,11 +1213,11 @@ __device__ __noinline__ void worker_w(const Ctx &c, const WorkerId &id)
             if (kk < nSp && ok) ok = warp_wait(c, bKFull + kk, 0);
             if (ok) ok = warp_wait(c, bVFull + k, 0);
             if (!ok) continue;
+            trace(c, 0x800 + k);
             uint32_t d[4][NW];
             load_rows<RP, false>(c, id, 0, c.buf(kb), d);
-            float2 kf[4][NW];
             float sr[4];
-            row_sums<NW>(d, w2, kf, sr);
+            row_sums<NW>(d, w2, sr);
             // value rows times 1/s_j (0 for rows without mass): hi part in place now, lo part once the hi-part MMAs have
             // read the buffer
             uint8_t *vt = c.buf(vb);
@@ -1223,10 +1256,12 @@ __device__ __noinline__ void worker_w(const Ctx &c, const WorkerId &id)
             }
             fence_proxy_async_smem();
             warp_arrive(c, bVLo + id.quad);
+            trace(c, 0x900 + k);
         }
         // ---- this segment's accumulator: pivot rows 16 w4 .. + 15 sit in the first 16 lanes of lane quarter w4; quad q
         // takes channels 32 q .. + 31.  The partial leaves multiplied by the key-side weights w2_t.
         if (ok) ok = warp_wait(c, bWFull + j, 0);
+        trace(c, 0xa00 + j);
         float v[16];
         if (ok) {
             tc_fence_after();
@@ -1256,7 +1291,7 @@ __device__ __noinline__ void worker_w(const Ctx &c, const WorkerId &id)
 
 // ---- phase O: the blocks of a slice add up W, then out = K~1 W'' / s_i per query tile
 template <int RP>
-__device__ __noinline__ void worker_o(const Ctx &c, const WorkerId &id)
+__device__ __noinline__ void worker_o(const Ctx c, const WorkerId id)
 {
     constexpr int NW = RP / 8;
     const ResParams &P = c.P;
@@ -1279,7 +1314,7 @@ __device__ __noinline__ void worker_o(const Ctx &c, const WorkerId &id)
                     if (c.M->abort) break;
                     const uint64_t now = global_timer_ns();
                     if (t0 == 0) t0 = now;
-                    else if (now - t0 > P.wait_ns) { c.M->abort = 1; record_timeout(c, 110 + j); raise_flag(P, 4 /* LOT_DEV_TIMEOUT */); break; }
+                    else if (now - t0 > P.wait_ns) { c.M->abort = 1; record_timeout(&P, c.M, c.warp, 110 + j); raise_flag(P, 4 /* LOT_DEV_TIMEOUT */); break; }
                 }
                 __nanosleep(32);
             }
@@ -1325,6 +1360,7 @@ __device__ __noinline__ void worker_o(const Ctx &c, const WorkerId &id)
     }
     fence_proxy_async_smem();
     named_bar_sync(1, kWorkers);
+    trace(c, 0xb00);
 
     const bool storer = id.w4 == 0 && c.lane == 0;
     for (int qq = id.quad; qq < M->nQ; qq += 2) {
@@ -1342,9 +1378,8 @@ __device__ __noinline__ void worker_o(const Ctx &c, const WorkerId &id)
         for (int e = 0; e < NW; ++e) w2[e] = *reinterpret_cast<const float2 *>(c.sW + sg * 64 + word_col<RP, true>(id, e));
         uint32_t d[4][NW];
         load_rows<RP, true>(c, id, id.lane_addr + qq * (RP / 2), nullptr, d);
-        float2 kf[4][NW];
         float sr[4];
-        row_sums<NW>(d, w2, kf, sr);
+        row_sums<NW>(d, w2, sr);
         // the tile as A operand: K-major rows of 64 bf16 (only the first RP columns are read)
 #pragma unroll
         for (int jj = 0; jj < 4; ++jj) {
@@ -1356,9 +1391,11 @@ __device__ __noinline__ void worker_o(const Ctx &c, const WorkerId &id)
         }
         fence_proxy_async_smem();
         warp_arrive(c, bAFull + id.quad);
+        trace(c, 0xc00 + qq);
         if (ok) ok = warp_wait(c, bOFull + id.quad, j & 1);
         if (!ok) continue;
         tc_fence_after();
+        trace(c, 0xd00 + qq);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             float o[32];
@@ -1409,11 +1446,11 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
 // Between two phases (one thread; nobody touches a barrier meanwhile, and every barrier is between two of its phases):
 // a barrier that has completed an odd number of phases gets one more full set of arrivals, so that the next phase of
 // the kernel finds every barrier as after its initialisation.
-__device__ __noinline__ void settle_bars(const Ctx &c)
+__device__ __noinline__ void settle_bars(uint32_t bar0)
 {
     for (int i = 0; i < bCount; ++i)
-        if (mbar_test_wait(c.bar(i), 0))
-            for (int a = 0; a < bar_count(i); ++a) mbar_arrive(c.bar(i));
+        if (mbar_test_wait(bar0 + 8 * i, 0))
+            for (int a = 0; a < bar_count(i); ++a) mbar_arrive(bar0 + 8 * i);
 }
 
 template <int RP>
@@ -1441,10 +1478,13 @@ resident_forward_kernel(const __grid_constant__ ResParams P)
     id.wtid = (int)threadIdx.x - 128;
     GatherState gs;
 
+    // time stamps of this block's phases (nanoseconds of the global timer), for profiling: [block][8] behind the records
+    unsigned long long *stamps = P.status + 2 + (size_t)gridDim.x * 12 + (size_t)blockIdx.x * 8;
+    if (threadIdx.x == 0) stamps[0] = global_timer_ns();
     auto phase_sync = [&](int next_phase) {
         tc_fence_before();
         __syncthreads();
-        if (threadIdx.x == 0) { settle_bars(c); c.M->phase = next_phase; }
+        if (threadIdx.x == 0) { settle_bars(c.bar(0)); c.M->phase = next_phase; if (next_phase <= kPhaseO) stamps[next_phase + 1] = global_timer_ns(); }
         __syncthreads();
         tc_fence_after();
     };
@@ -1456,9 +1496,10 @@ resident_forward_kernel(const __grid_constant__ ResParams P)
                 for (int i = 0; i < bCount; ++i) mbar_init(c.bar(i), bar_count(i));
                 fence_barrier_init();
             } else {
-                settle_bars(c);
+                settle_bars(c.bar(0));
             }
             c.M->phase = kPhaseX;
+            stamps[1] = global_timer_ns();
         }
         for (int i = threadIdx.x; i < kMaxSeg * 64; i += kThreads) c.sW[i] = (i & 63) < P.r ? 1.f : 0.f;
         tc_fence_before();
@@ -1491,9 +1532,9 @@ resident_forward_kernel(const __grid_constant__ ResParams P)
         else worker_x<RP>(c, id);
         phase_sync(kPhaseS);
         // ---------------- phase S
+        if (warp == 0 && c.lane == 0) producer_s(c);
         if (P.T > 1) {
-            if (warp == 0) { if (c.lane == 0) producer_s(c); }
-            else if (warp == 2) publisher<RP>(c, 1, P.T);
+            if (warp == 2) publisher<RP>(c, 1, P.T);
             else if (warp == 3) gatherer<RP>(c, gs, 1, P.T);
             else if (warp >= 4) worker_s<RP>(c, id);
         }
@@ -1509,6 +1550,7 @@ resident_forward_kernel(const __grid_constant__ ResParams P)
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
+        if (threadIdx.x == 0) stamps[5] = global_timer_ns();
     }
     if (warp == 1) tmem_dealloc(c.M->tmem, 512);
 }
@@ -1568,6 +1610,7 @@ static inline int pad_r(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
 static std::atomic<unsigned> g_tag{0x1000u};
 static std::atomic<long long> g_wait_ns{1000000000ll};
 static std::atomic<int> g_skip_cta{-1};
+static std::atomic<unsigned long long *> g_trace{nullptr};
 
 } // namespace resident
 
@@ -1588,6 +1631,7 @@ void resident_debug(int what, long long value)
 {
     if (what == 1) resident::g_skip_cta.store((int)value);
     else if (what == 2) resident::g_wait_ns.store(value > 0 ? value : 1000000000ll);
+    else if (what == 3) resident::g_trace.store(reinterpret_cast<unsigned long long *>(value));
 }
 
 ResidentGeom resident_geometry(int dtype, int B, int H, int n, int d, int r)
@@ -1633,7 +1677,8 @@ ResidentLayout resident_layout(int B, int H, int n, int d, int r)
     const size_t BH = (size_t)B * H;
     const int RP = pad_r(r);
     size_t o = 0;
-    L.status = o; o += up256(16 + (size_t)G.ctas * 12 * 8);   // status word, redo word at + 8, then one record per warp of a wait that gave up
+    // status word, redo word at + 8, then one record per warp of a wait that gave up, then eight time stamps per block
+    L.status = o; o += up256(16 + (size_t)G.ctas * 12 * 8 + (size_t)G.ctas * 8 * 8);
     L.part = o; o += up256((size_t)2 * 2 * BH * G.maxslots * RP * 8);
     L.wflag = o; o += up256(BH * G.maxslots * 8);
     L.wpart = o; o += up256(BH * G.maxslots * 64 * kDK * 4);
@@ -1694,6 +1739,7 @@ cudaError_t resident_attention(const void *q, const void *k, const void *v, cons
     P.eps_ln2 = (float)((double)eps * 0.6931471805599453);
     P.wait_ns = (unsigned long long)g_wait_ns.load();
     P.skip_publish_cta = g_skip_cta.exchange(-1);
+    P.trace = g_trace.load();
     *tag_out = P.tag;
 
     const int RP = pad_r(r);

@@ -23,7 +23,8 @@ def gpu_forward(x, want_g=False):
     out, ws = lot.lot_attention_fwd_ex(t["q"], t["k"], t["v"], t["z"], t["beta"], t["key_len"], x.eps, x.iters,
                                        g1_out=g1, g2_out=g2)
     torch.cuda.synchronize()
-    status = lot.lot_device_status(ws)
+    # LOT_DEV_RECOMPUTED is information, not an error: whichever tensor-core kernel produced the result, it is checked
+    status = lot.lot_device_status(ws) & ~lot.LOT_DEV_RECOMPUTED
     res = dict(out=out.float().cpu().double().numpy(), status=status)
     if want_g:
         res["g1"] = g1.cpu().double().numpy()

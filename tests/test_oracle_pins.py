@@ -298,3 +298,131 @@ def test_golden_config1_matches_stored_oracle_values():
     x = synth.config(1); d = x.f64()
     out = O.attention_fwd(d["q"], d["k"], d["v"], d["z"], d["beta"], x.eps, x.iters)
     np.testing.assert_allclose(out[0, 0, ::8, :], stored, rtol=0, atol=1e-13)
+
+
+# ================================================================ forward variants and the gradient
+# (Section "Empirical measures and pivot": arbitrary weights; Appendix "Bidirectional scope": cross-attention;
+#  Eq. (5): the [CLS] row; Section "Learning": back-propagation through the two solves and the composition)
+from oracle import lot_oracle_grad as OG
+
+
+def _rand_head(rng, nq, nk, d, dv, r):
+    q, k, v, z = rng.normal(size=(nq, d)) * 0.6, rng.normal(size=(nk, d)) * 0.6, rng.normal(size=(nk, dv)), rng.normal(size=(r, d))
+    beta = rng.random(r) + 0.2; beta /= beta.sum()
+    a = rng.random(nq) + 0.1; a /= a.sum()
+    b = rng.random(nk) + 0.1; b /= b.sum()
+    return q, k, v, z, beta, a, b
+
+
+def test_warm_start_continues_the_iteration():
+    """T1 iterations, then T2 more from the exported pivot potential, are T1 + T2 iterations: the potential is the
+    whole state between two passes."""
+    rng = np.random.default_rng(3)
+    C = rng.normal(size=(37, 5)); beta = np.full(5, 0.2); m = np.full(37, 1 / 37)
+    g_a, _, _ = O.sinkhorn(C, beta, m, 0.3, 4)
+    g_b, f_b, P_b = O.sinkhorn_from(C, beta, m, 0.3, 7, g_a)
+    g_c, f_c, P_c = O.sinkhorn(C, beta, m, 0.3, 11)
+    np.testing.assert_allclose(g_b, g_c, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(P_b, P_c, rtol=0, atol=1e-15)
+    # and a start at the fixed point stays there
+    g_inf, _, P_inf = O.sinkhorn(C, beta, m, 0.3, 3000)
+    g_again, _, P_again = O.sinkhorn_from(C, beta, m, 0.3, 1, g_inf)
+    np.testing.assert_allclose(P_again, P_inf, rtol=0, atol=1e-14)
+
+
+def test_cross_attention_and_general_marginals_by_brute_force():
+    """nq != nk with arbitrary weights: at convergence the explicit nq x nk coupling has row sums a and column sums b
+    to 1e-9 and rank <= r; the factorised output equals Diag(1/a) Gamma V; equal sizes and uniform weights reduce to
+    the square routine."""
+    rng = np.random.default_rng(11)
+    q, k, v, z, beta, a, b = _rand_head(rng, 23, 31, 6, 4, 5)
+    h = O.head_x(q, k, v, z, beta, a, b, 0.4, 5000)
+    G = O.coupling(h["P1"], h["P2"], beta)
+    assert np.abs(G.sum(1) - a).max() < 1e-9 and np.abs(G.sum(0) - b).max() < 1e-9
+    sv = np.linalg.svd(G, compute_uv=False)
+    assert sv[5] / sv[0] < 1e-12
+    np.testing.assert_allclose(h["out"], (G / a[:, None]) @ v, atol=1e-12)
+    # a key with zero weight is out of the problem: the same as deleting it
+    b0 = b.copy(); b0[7] = 0; b0 /= b0.sum()
+    h0 = O.head_x(q, k, v, z, beta, a, b0, 0.4, 50)
+    keep = np.arange(31) != 7
+    h1 = O.head_x(q, k[keep], v[keep], z, beta, a, b0[keep], 0.4, 50)
+    np.testing.assert_allclose(h0["out"], h1["out"], atol=1e-13)
+    # square and uniform: the routine the configurations use
+    n = 19
+    q2, k2, v2 = rng.normal(size=(n, 6)), rng.normal(size=(n, 6)), rng.normal(size=(n, 6))
+    u = np.full(n, 1 / n)
+    np.testing.assert_allclose(O.head_x(q2, k2, v2, z, beta, u, u, 0.4, 9)["out"], O.head(q2, k2, v2, z, beta, u, u, 0.4, 9)["out"],
+                               atol=1e-14)
+
+
+def test_cls_row_is_a_library_softmax_and_the_rest_is_the_smaller_problem():
+    from scipy.special import softmax
+    rng = np.random.default_rng(5)
+    n, d, r, tau = 17, 8, 4, 1.7
+    q, k, v, z = rng.normal(size=(n, d)), rng.normal(size=(n, d)), rng.normal(size=(n, d)), rng.normal(size=(r, d))
+    beta = np.array([0.1, 0.2, 0.3, 0.4])
+    out = O.head_cls(q, k, v, z, beta, 0.5, 12, tau)
+    np.testing.assert_allclose(out[0], softmax(tau * (k @ q[0])) @ v, atol=1e-13)
+    u = np.full(n - 1, 1 / (n - 1))
+    np.testing.assert_allclose(out[1:], O.head(q[1:], k[1:], v[1:], z, beta, u, u, 0.5, 12)["out"], atol=1e-13)
+    # a constant value vector comes back unchanged in every row: each row of the implied attention matrix sums to 1
+    ones = O.head_cls(q, k, np.ones((n, 3)), z, beta, 0.5, 400, tau)
+    np.testing.assert_allclose(ones, 1.0, atol=1e-9)
+    # key mask: the softmax row and the transport problem both leave the padded keys out
+    outm = O.head_cls(q, k, v, z, beta, 0.5, 12, tau, key_len=11)
+    np.testing.assert_allclose(outm[0], softmax(tau * (k[:11] @ q[0])) @ v[:11], atol=1e-13)
+
+
+def test_gradient_forward_agrees_with_the_c_oracle():
+    rng = np.random.default_rng(2)
+    q, k, v, z, beta, a, b = _rand_head(rng, 11, 13, 5, 3, 4)
+    g10, g20 = rng.normal(size=4) * 0.1, rng.normal(size=4) * 0.1
+    fw = OG.head_forward(q, k, v, z, beta, a, b, 0.35, 6, g10, g20)
+    ref = O.head_x(q, k, v, z, beta, a, b, 0.35, 6, g10, g20)
+    np.testing.assert_allclose(fw["out"], ref["out"], atol=1e-13)
+    np.testing.assert_allclose(fw["g1"], ref["g1"], atol=1e-13)
+    np.testing.assert_allclose(fw["P2"], ref["P2"], atol=1e-14)
+
+
+@pytest.mark.parametrize("iters", [0, 1, 5])
+def test_gradient_matches_central_differences(iters):
+    """Every input's gradient against central finite differences of the C oracle's forward (a dropped term, a wrong
+    sign or a transposed factor in the reverse sweep fails here)."""
+    rng = np.random.default_rng(7 + iters)
+    q, k, v, z, beta, a, b = _rand_head(rng, 7, 9, 4, 3, 3)
+    dout = rng.normal(size=(7, 3))
+    eps = 0.45
+    g10, g20 = rng.normal(size=3) * 0.2, rng.normal(size=3) * 0.2
+    grads = OG.head_backward(OG.head_forward(q, k, v, z, beta, a, b, eps, iters, g10, g20), dout)
+
+    def loss(**kw):
+        args = dict(q=q, k=k, v=v, z=z, beta=beta, g1_0=g10, g2_0=g20)
+        args.update(kw)
+        return float(np.sum(O.head_x(args["q"], args["k"], args["v"], args["z"], args["beta"], a, b, eps, iters,
+                                     args["g1_0"], args["g2_0"])["out"] * dout))
+
+    h = 1e-6
+    for name, x0 in (("q", q), ("k", k), ("v", v), ("z", z), ("beta", beta), ("g1_0", g10), ("g2_0", g20)):
+        fd = np.zeros_like(x0)
+        it = np.nditer(x0, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            xp, xm = x0.copy(), x0.copy()
+            xp[idx] += h; xm[idx] -= h
+            fd[idx] = (loss(**{name: xp}) - loss(**{name: xm})) / (2 * h)
+        got = grads["d" + name]
+        assert np.abs(got - fd).max() <= 2e-6 * max(1.0, np.abs(fd).max()), name
+
+
+def test_gradient_at_convergence_forgets_the_starting_potential():
+    """At the fixed point the result no longer depends on where the iteration started: the gradient with respect to
+    the starting potentials vanishes, and the other gradients agree for two different starts."""
+    rng = np.random.default_rng(19)
+    q, k, v, z, beta, a, b = _rand_head(rng, 8, 8, 4, 3, 3)
+    dout = rng.normal(size=(8, 3))
+    g_a = OG.head_backward(OG.head_forward(q, k, v, z, beta, a, b, 0.5, 400), dout)
+    g_b = OG.head_backward(OG.head_forward(q, k, v, z, beta, a, b, 0.5, 400, rng.normal(size=3), rng.normal(size=3)), dout)
+    assert np.abs(g_a["dg1_0"]).max() < 1e-12 and np.abs(g_b["dg2_0"]).max() < 1e-12
+    for name in ("dq", "dk", "dv", "dz", "dbeta"):
+        np.testing.assert_allclose(g_a[name], g_b[name], atol=1e-10)
