@@ -206,6 +206,35 @@ LOT_API int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
                          void *out, float *g1_out, float *g2_out,
                          void *ws, size_t ws_bytes, lot_stream_t stream);
 
+/* Scratch bytes lot_attention_fwd_var needs for these sizes. */
+LOT_API size_t lot_var_workspace_bytes(int B, int H, int nq, int nk, int d, int r, int dtype);
+
+/*
+ * lot_attention_fwd_var -- the forward path with the variations the paper uses around it:
+ *   cross-attention   nq queries, nk keys and values per slice (Appendix "Bidirectional scope", closing
+ *                     paragraph): q, out [B,H,nq,d];  k, v [B,H,nk,d].
+ *   token weights     a [B,H,nq], b [B,H,nk] float32 or NULL: the weights p^1, p^2 of the empirical measures
+ *                     (Section "Empirical measures and pivot"; >= 0, each slice summing to 1, trusted).  NULL
+ *                     means uniform, over the first key_len[b] keys on the key side when key_len is given.  A
+ *                     token of weight zero takes no part in its transport problem; a query of weight zero gets
+ *                     an all-zero output row.  out = Diag(1/a) Gamma1^T Diag(1/beta) Gamma2 V.
+ *   warm start        g1_in, g2_in [B,H,r] float32 or NULL: pivot potentials (natural-log units, as g1_out and
+ *                     g2_out give them) the two iterations start from instead of zero.  T1 iterations followed
+ *                     by T2 more from the exported potentials are T1 + T2 iterations.
+ *   [CLS] row         cls = 1 (Eq. (5)): token 0 is the class token.  Its output row is the plain softmax
+ *                     aggregate sum_j softmax_j(cls_tau <q_0, k_j>) v_j over all valid keys (cls_tau > 0 is the
+ *                     temperature the paper calls beta in Eq. (5)); every other row follows the transport rule
+ *                     among the remaining tokens (queries 1.., valid keys 1.., uniform weights).  a and b must
+ *                     be NULL; nq, nk >= 2 are needed for the transport part (else LOT_DEV_EMPTY is flagged).
+ * Everything else as lot_attention_fwd_ex.  This entry point runs on the general path for every shape.
+ */
+LOT_API int lot_attention_fwd_var(const void *q, const void *k, const void *v, const float *z, const float *beta,
+                          const float *a, const float *b, const int32_t *key_len,
+                          const float *g1_in, const float *g2_in, int cls, float cls_tau,
+                          int dtype, int B, int H, int nq, int nk, int d, int r, float eps, int iters,
+                          void *out, float *g1_out, float *g2_out,
+                          void *ws, size_t ws_bytes, lot_stream_t stream);
+
 /*
  * lot_attention_fwd -- the same path for float32 tensors, uniform marginals, with scratch the
  * library manages itself: one buffer per device, grown with cudaMalloc when a call needs

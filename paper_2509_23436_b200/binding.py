@@ -36,6 +36,8 @@ SIGNATURES = {
     "lot_launch_count": (_i, [_i, _i, _i, _i, _i, _i, _i]),
     "lot_attention_fwd_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _f, _i,
                                   _vp, _vp, _vp, _vp, _sz, _vp]),
+    "lot_var_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
+    "lot_attention_fwd_var": (_i, [_vp] * 10 + [_i, _f] + [_i] * 7 + [_f, _i] + [_vp, _vp, _vp, _vp, _sz, _vp]),
     "lot_attention_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp]),
     "lot_device_status": (_i, [_vp, _vp, ctypes.POINTER(_i)]),
 }
@@ -183,6 +185,37 @@ def lot_attention_fwd_ex(q, k, v, z, beta, key_len, eps, iters, *, out=None, g1_
                                     _dev(g2_out, "g2_out", torch.float32),
                                     _dev(ws, "ws"), ws.numel(), _stream(stream))
     _check(st, "lot_attention_fwd_ex")
+    return out, ws
+
+
+def lot_var_workspace_bytes(B, H, nq, nk, d, r, dtype_code) -> int:
+    return lib().lot_var_workspace_bytes(B, H, nq, nk, d, r, dtype_code)
+
+
+def lot_attention_fwd_var(q, k, v, z, beta, eps, iters, *, a=None, b=None, key_len=None, g1_in=None, g2_in=None,
+                          cls=False, cls_tau=1.0, out=None, g1_out=None, g2_out=None, ws=None, stream=None):
+    """Forward variants (cross-attention, token weights, warm start, [CLS] row).  Returns (out, ws)."""
+    B, H, nq, d = q.shape
+    nk = k.shape[2]
+    r = z.shape[1]
+    code = _dtype_code(q)
+    if k.shape != (B, H, nk, d) or v.shape != k.shape or k.dtype != q.dtype or v.dtype != q.dtype:
+        raise LotError("k, v must be [B,H,nk,d] in q's dtype")
+    if tuple(z.shape) != (H, r, d) or tuple(beta.shape) != (H, r):
+        raise LotError("z must be [H,r,d] and beta [H,r]")
+    if out is None:
+        out = torch.empty_like(q)
+    need = lot_var_workspace_bytes(B, H, nq, nk, d, r, code)
+    if ws is None:
+        ws = torch.empty(max(need, 256), device=q.device, dtype=torch.uint8)
+    f32 = torch.float32
+    st = lib().lot_attention_fwd_var(_dev(q, "q"), _dev(k, "k"), _dev(v, "v"), _dev(z, "z", f32), _dev(beta, "beta", f32),
+                                     _dev(a, "a", f32), _dev(b, "b", f32), _dev(key_len, "key_len", torch.int32),
+                                     _dev(g1_in, "g1_in", f32), _dev(g2_in, "g2_in", f32), int(bool(cls)), float(cls_tau),
+                                     code, B, H, nq, nk, d, r, float(eps), int(iters),
+                                     _dev(out, "out", q.dtype), _dev(g1_out, "g1_out", f32), _dev(g2_out, "g2_out", f32),
+                                     _dev(ws, "ws"), ws.numel(), _stream(stream))
+    _check(st, "lot_attention_fwd_var")
     return out, ws
 
 

@@ -89,6 +89,38 @@ AttnLayout attn_layout(int B, int H, int n, int d, int r, int dtype)
     return A;
 }
 
+// Workspace of lot_attention_fwd_var: the two sides have their own token counts, so each gets a Sinkhorn block.
+struct VarLayout {
+    SinkLayout s1, s2;
+    size_t counter2, cost1, cost2, wa, wb, scores, wpart, Wp, total;
+    int achunks, arows;
+};
+
+VarLayout var_layout(int B, int H, int nq, int nk, int d, int r, int dtype)
+{
+    VarLayout V;
+    const size_t lt = dtype == LOT_F32 ? 8 : 4;
+    const int BH = B * H;
+    const int tiles = ((r + 63) / 64) * ((d + 63) / 64) * BH;
+    V.counter2 = 256;
+    size_t o = 256 + up256((size_t)tiles * 4);
+    // one cleared head for both sides: status word at 0, then tickets and potentials
+    V.s1 = sink_layout(BH, nq, r, o, lt);
+    V.s2 = sink_layout(BH, nk, r, V.s1.total, lt);
+    o = V.s2.total;
+    V.cost1 = o; o += up256((size_t)BH * nq * r * lt);
+    V.cost2 = o; o += up256((size_t)BH * nk * r * lt);
+    V.wa = o; o += up256((size_t)BH * nq * 4);
+    V.wb = o; o += up256((size_t)BH * nk * 4);
+    V.scores = o; o += up256((size_t)BH * nk * 4);
+    V.achunks = apply_chunks(BH > 0 ? BH : 1, nk > 0 ? nk : 1, r, d);
+    V.arows = (nk + V.achunks - 1) / V.achunks;
+    V.wpart = o; o += up256((size_t)BH * V.achunks * r * d * 4);
+    V.Wp = o; o += up256((size_t)BH * r * d * 4);
+    V.total = o;
+    return V;
+}
+
 template <typename T> inline T *at(void *ws, size_t off) { return reinterpret_cast<T *>(static_cast<char *>(ws) + off); }
 
 struct Managed {
@@ -362,7 +394,7 @@ int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
     ap.M1 = a.M; ap.M2 = static_cast<char *>(a.M) + (size_t)BH * n * lt;
     ap.beta = beta; ap.key_len = key_len; ap.v = v; ap.out = out;
     ap.wpart = at<float>(ws, A.wpart); ap.Wp = at<float>(ws, A.Wp); ap.counter = at<unsigned>(ws, A.counter2);
-    ap.B = B; ap.H = H; ap.n = n; ap.d = d; ap.r = r;
+    ap.B = B; ap.H = H; ap.n = n; ap.nk = n; ap.d = d; ap.r = r;
     ap.chunks = A.achunks; ap.rows_per_chunk = A.arows; ap.scale_d = a.scale_d;
     if (launch_apply_w(ap, dtype, s) != cudaSuccess) return LOT_ERR_CUDA;
     if (launch_apply_out(ap, dtype, s) != cudaSuccess) return LOT_ERR_CUDA;
@@ -371,6 +403,99 @@ int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
     if (g1_out && cudaMemcpyAsync(g1_out, a.g_out, gb, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LOT_ERR_CUDA;
     if (g2_out && cudaMemcpyAsync(g2_out, a.g_out + (size_t)BH * r, gb, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
         return LOT_ERR_CUDA;
+    return LOT_OK;
+}
+
+size_t lot_var_workspace_bytes(int B, int H, int nq, int nk, int d, int r, int dtype)
+{
+    if (dtype != LOT_F32 && dtype != LOT_BF16) return 0;
+    if (check_dims(B, H, nq, r) != LOT_OK || check_dims(B, H, nk, r) != LOT_OK) return 0;
+    if (check_d(nq, d) != LOT_OK || check_d(nk, d) != LOT_OK) return 0;
+    return var_layout(B, H, nq, nk, d, r, dtype).total;
+}
+
+int lot_attention_fwd_var(const void *q, const void *k, const void *v, const float *z, const float *beta,
+                          const float *a, const float *b, const int32_t *key_len,
+                          const float *g1_in, const float *g2_in, int cls, float cls_tau,
+                          int dtype, int B, int H, int nq, int nk, int d, int r, float eps, int iters,
+                          void *out, float *g1_out, float *g2_out,
+                          void *ws, size_t ws_bytes, lot_stream_t stream)
+{
+    if (dtype != LOT_F32 && dtype != LOT_BF16) return LOT_ERR_INVALID_ARG;
+    int st = check_dims(B, H, nq, r);
+    if (st == LOT_OK) st = check_dims(B, H, nk, r);
+    if (st == LOT_OK) st = check_d(nq, d);
+    if (st == LOT_OK) st = check_d(nk, d);
+    if (st != LOT_OK) return st;
+    if (!(eps > 0.f) || !isfinite(eps) || iters < 0) return LOT_ERR_INVALID_ARG;
+    if (cls != 0 && cls != 1) return LOT_ERR_INVALID_ARG;
+    if (cls && (!(cls_tau > 0.f) || !isfinite(cls_tau) || a != nullptr || b != nullptr)) return LOT_ERR_INVALID_ARG;
+    if (B == 0 || nq == 0) return LOT_OK;
+    if (nk == 0) return LOT_ERR_INVALID_ARG;
+    if (!q || !k || !v || !z || !beta || !out) return LOT_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(z) || !aligned16(beta) || !aligned16(out) ||
+        !aligned16(g1_out) || !aligned16(g2_out) || !aligned16(g1_in) || !aligned16(g2_in) || !aligned16(a) ||
+        !aligned16(b) || (key_len && (reinterpret_cast<uintptr_t>(key_len) & 3u)))
+        return LOT_ERR_INVALID_ARG;
+    VarLayout V = var_layout(B, H, nq, nk, d, r, dtype);
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < V.total) return LOT_ERR_WORKSPACE;
+    const bool wide = dtype == LOT_F32;
+    const size_t lt = wide ? 8 : 4;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int BH = B * H;
+    remember_ws(ws, kPathGeneral, 0, 0);
+    // the head (status word, tickets) starts at zero; the potentials start at the given ones
+    if (cudaMemsetAsync(ws, 0, V.s1.head_end, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (cudaMemsetAsync(at<char>(ws, V.s2.status), 0, V.s2.head_end - V.s2.status, s) != cudaSuccess) return LOT_ERR_CUDA;
+    const double scale = 1.4426950408889634 / (double)eps;
+    if (g1_in && launch_g_init(g1_in, at<void>(ws, V.s1.G), (size_t)BH * r, scale, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (g2_in && launch_g_init(g2_in, at<void>(ws, V.s2.G), (size_t)BH * r, scale, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    const float *wa = a, *wb = b;
+    if (cls) {
+        if (launch_cls_marginals(at<float>(ws, V.wa), at<float>(ws, V.wb), key_len, B, H, nq, nk, at<int>(ws, 0), s) != cudaSuccess)
+            return LOT_ERR_CUDA;
+        wa = at<float>(ws, V.wa);
+        wb = at<float>(ws, V.wb);
+    }
+
+    char *cost1 = at<char>(ws, V.cost1), *cost2 = at<char>(ws, V.cost2);
+    if (launch_cost(q, z, dtype, BH, H, nq, d, r, cost1, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_cost(k, z, dtype, BH, H, nk, d, r, cost2, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+
+    PassArgs pa[2];
+    for (int side = 0; side < 2; ++side) {
+        const SinkLayout &L = side ? V.s2 : V.s1;
+        PassArgs &x = pa[side];
+        x = PassArgs{};
+        x.cost = side ? cost2 : cost1; x.beta = beta;
+        // a key length is a mask on the key side only; with explicit weights it only bounds the rows that are read
+        x.len = side ? key_len : nullptr; x.len_from = 0;
+        x.mass = side ? wb : wa;
+        x.G = at<void>(ws, L.G); x.part = at<float>(ws, L.part); x.counter = at<unsigned>(ws, L.counter);
+        x.M = at<void>(ws, L.M); x.g_out = side ? g2_out : g1_out;
+        x.status = at<int>(ws, 0);
+        x.nprob = BH; x.B = B; x.H = H; x.n = side ? nk : nq; x.r = r;
+        x.chunks = L.chunks; x.rows_per_chunk = L.rows_per_chunk;
+        x.mode = wide ? kModeWide : kModeF32;
+        x.scale_d = scale;
+        x.eps_ln2 = (float)((double)eps * 0.6931471805599453);
+        for (int it = 0; it < iters; ++it)
+            if (launch_sinkhorn_pass(x, false, s) != cudaSuccess) return LOT_ERR_CUDA;
+        if (launch_sinkhorn_pass(x, true, s) != cudaSuccess) return LOT_ERR_CUDA;
+    }
+
+    ApplyArgs ap{};
+    ap.cost1 = cost1; ap.cost2 = cost2;
+    ap.G1 = pa[0].G; ap.G2 = pa[1].G; ap.M1 = pa[0].M; ap.M2 = pa[1].M;
+    ap.beta = beta; ap.key_len = key_len; ap.mass2 = wb; ap.v = v; ap.out = out;
+    ap.wpart = at<float>(ws, V.wpart); ap.Wp = at<float>(ws, V.Wp); ap.counter = at<unsigned>(ws, V.counter2);
+    ap.B = B; ap.H = H; ap.n = nq; ap.nk = nk; ap.d = d; ap.r = r;
+    ap.chunks = V.achunks; ap.rows_per_chunk = V.arows; ap.scale_d = scale;
+    if (launch_apply_w(ap, dtype, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_apply_out(ap, dtype, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (cls && launch_cls_row(q, k, v, key_len, dtype, B, H, nq, nk, d, cls_tau, at<float>(ws, V.scores), out, s) != cudaSuccess)
+        return LOT_ERR_CUDA;
+    (void)lt;
     return LOT_OK;
 }
 

@@ -21,6 +21,8 @@ struct PassArgs {
     const float *beta;   // [H][r]
     const int32_t *len;  // [B] or nullptr
     int len_from;
+    const float *mass;   // [nprob][n] token weights (>= 0; zero takes the token out of the problem), or nullptr:
+                         // uniform over the valid tokens
     void *G;             // [nprob][r] pivot potentials, base-2 log units (in/out; float or double)
     float *part;         // [nprob][chunks][r][2] per-block column pairs (kappa, S)
     unsigned *counter;   // [nprob] arrival tickets, zero on entry and on exit
@@ -43,12 +45,14 @@ struct ApplyArgs {
     const void *M1, *M2;   // [BH][n]
     const float *beta;     // [H][r]
     const int32_t *key_len;
-    const void *v;         // [BH][n][d]
+    const float *mass2;    // [BH][nk] key weights or nullptr (uniform over the valid keys)
+    const void *v;         // [BH][nk][d]
     void *out;             // [BH][n][d]
     float *wpart;          // [BH][chunks][r][d]
     float *Wp;             // [BH][r][d]  W' = Diag(beta)^-1 Gamma2 V
     unsigned *counter;     // [BH * tblks * cblks]
-    int B, H, n, d, r;
+    int B, H, n, d, r;     // n: queries per slice
+    int nk;                // keys per slice
     int chunks, rows_per_chunk;
     double scale_d;
 };
@@ -61,6 +65,14 @@ cudaError_t launch_cost(const void *x, const float *z, int dtype, int BH, int H,
 cudaError_t launch_sinkhorn_pass(const PassArgs &a, bool final_pass, cudaStream_t st);
 cudaError_t launch_apply_w(const ApplyArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_apply_out(const ApplyArgs &a, int dtype, cudaStream_t st);
+// starting potentials: G = g_in * scale (float or double per `wide`), zeros when g_in == nullptr
+cudaError_t launch_g_init(const float *g_in, void *G, size_t count, double scale, bool wide, cudaStream_t st);
+// weights of the [CLS] treatment, Eq. (5): a = (0, 1/(nq-1), ...), b = (0, 1/(kv-1), ... up to the key length, 0 ...)
+cudaError_t launch_cls_marginals(float *a, float *b, const int32_t *key_len, int B, int H, int nq, int nk, int *status,
+                                 cudaStream_t st);
+// row 0 of every slice: softmax_j(tau <q_0, k_j>) over the valid keys, applied to v; scores: [BH][nk] scratch
+cudaError_t launch_cls_row(const void *q, const void *k, const void *v, const int32_t *key_len, int dtype, int B, int H,
+                           int nq, int nk, int d, float tau, float *scores, void *out, cudaStream_t st);
 
 // ---- fused tensor-core path (lot_fused.cu): bf16 tensors, d = 64, r <= 64 ----
 struct FusedLayout {

@@ -120,6 +120,7 @@ sinkhorn_pass_kernel(PassArgs a)
     LT *Gp = static_cast<LT *>(a.G) + (size_t)p * r;
     LT *Mp = static_cast<LT *>(a.M) + (size_t)p * a.n;
     const LT scale = (LT)a.scale_d;
+    const float *mass_p = a.mass ? a.mass + (size_t)p * a.n : nullptr;
 
     LT Gk[CPL];
     float kap[CPL], S[CPL];
@@ -141,7 +142,9 @@ sinkhorn_pass_kernel(PassArgs a)
 
     for (int base = row0 + warp * RPW; base < loop_end; base += kPassWarps * RPW) {
         const int i = base + sub;
-        const bool rv = i < row1;
+        const float mi = (mass_p != nullptr && i < row1) ? __ldg(mass_p + i) : mass;
+        const bool rv = i < row1 && mi > 0.f;
+        const float lmi = mass_p != nullptr ? lg2(mi) : log2m;      // log2 of this token's weight
         LT l[CPL];
         LT m = (LT)neg_inf();
 #pragma unroll
@@ -166,19 +169,19 @@ sinkhorn_pass_kernel(PassArgs a)
             if (rv) {
 #pragma unroll
                 for (int k = 0; k < CPL; ++k)
-                    if (cv[k]) pair_add(kap[k], S[k], e[k] - lgs);
+                    if (cv[k]) pair_add(kap[k], S[k], mass_p != nullptr ? e[k] - lgs + lmi : e[k] - lgs);
             }
         } else if (i < row_end) {
             if (cl == 0) {
                 const LT Mi = m + (LT)lgs;
                 Mp[i] = rv ? Mi : (LT)__int_as_float(0x7f800000);
-                if (a.f_out) a.f_out[(size_t)p * a.n + i] = rv ? (float)((LT)a.eps_ln2 * ((LT)log2m - Mi)) : neg_inf();
+                if (a.f_out) a.f_out[(size_t)p * a.n + i] = rv ? (float)((LT)a.eps_ln2 * ((LT)lmi - Mi)) : neg_inf();
             }
             if (a.plan_out) {
 #pragma unroll
                 for (int k = 0; k < CPL; ++k)
                     if (cv[k])
-                        a.plan_out[((size_t)p * a.n + i) * r + cl + k * GS] = rv ? mass * ex2(e[k] - lgs) : 0.f;
+                        a.plan_out[((size_t)p * a.n + i) * r + cl + k * GS] = rv ? mi * ex2(e[k] - lgs) : 0.f;
             }
         }
     }
@@ -235,7 +238,8 @@ sinkhorn_pass_kernel(PassArgs a)
             atomicOr(a.status, 2 /* LOT_DEV_EMPTY */);
         } else {
             LT lam = (LT)kk + (LT)lg2(ss);
-            LT gn = Gp[t] + (LT)lg2(a.beta[h * r + t] * (float)nvalid) - lam;
+            // uniform weights: the common factor 1/nvalid was left out of the column sums
+            LT gn = Gp[t] + (LT)lg2(a.mass ? a.beta[h * r + t] : a.beta[h * r + t] * (float)nvalid) - lam;
             if (!isfinite((float)gn)) atomicOr(a.status, 1 /* LOT_DEV_NONFINITE */);
             Gp[t] = gn;
         }
@@ -313,9 +317,10 @@ apply_w_kernel(ApplyArgs a)
     const int tblk = blockIdx.y / cblks, cblk = blockIdx.y % cblks;
     const int t0 = tblk * kTile, c0 = cblk * kTile;
     const int chunk = blockIdx.x;
-    const int n = a.n, r = a.r, d = a.d;
+    const int n = a.nk, r = a.r, d = a.d;
     int nvalid = n;
     if (a.key_len != nullptr) nvalid = min(max(a.key_len[b], 0), n);
+    const float *mass2 = a.mass2 ? a.mass2 + (size_t)bh * n : nullptr;
     const int row0 = chunk * a.rows_per_chunk;
     const int row1 = min(min(row0 + a.rows_per_chunk, n), nvalid);
     const LT *C = static_cast<const LT *>(a.cost2) + (size_t)bh * n * r;
@@ -333,7 +338,10 @@ apply_w_kernel(ApplyArgs a)
             int jj = idx / kTile, tt = idx % kTile;
             int j = j0 + jj, t = t0 + tt;
             float val = 0.f;
-            if (j < row1 && t < r) val = ex2((float)(fma(__ldg(C + (size_t)j * r + t), scale, __ldg(G + t)) - __ldg(M + j)));
+            if (j < row1 && t < r) {
+                val = ex2((float)(fma(__ldg(C + (size_t)j * r + t), scale, __ldg(G + t)) - __ldg(M + j)));
+                if (mass2 != nullptr) val *= __ldg(mass2 + j);        // a massless key has M = +inf: val is 0 already
+            }
             Ps[jj][tt] = val;
         }
 #pragma unroll
@@ -377,7 +385,7 @@ apply_w_kernel(ApplyArgs a)
     __syncthreads();
     if (!sm_last) return;
     __threadfence();
-    const float mass = nvalid > 0 ? 1.f / (float)nvalid : 0.f;
+    const float mass = a.mass2 ? 1.f : (nvalid > 0 ? 1.f / (float)nvalid : 0.f);
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
         int t = t0 + ty * 4 + x;
@@ -471,6 +479,120 @@ cudaError_t launch_apply_out(const ApplyArgs &a, int dtype, cudaStream_t st)
     dim3 grid((a.n + kTile - 1) / kTile, (a.d + kTile - 1) / kTile, a.B * a.H);
     if (dtype == 0) apply_out_kernel<float, double><<<grid, 256, 0, st>>>(a);
     else apply_out_kernel<__nv_bfloat16, float><<<grid, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------
+// Forward variants: starting potentials, the weights and the softmax row of the [CLS] treatment
+// ------------------------------------------------------------------------------------
+template <typename LT>
+__global__ void g_init_kernel(const float *__restrict__ g_in, LT *__restrict__ G, size_t count, double scale)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x)
+        G[i] = g_in ? (LT)((double)g_in[i] * scale) : (LT)0;
+}
+
+cudaError_t launch_g_init(const float *g_in, void *G, size_t count, double scale, bool wide, cudaStream_t st)
+{
+    if (count == 0) return cudaSuccess;
+    const int blocks = (int)((count + 255) / 256 < 1024 ? (count + 255) / 256 : 1024);
+    if (wide) g_init_kernel<double><<<blocks, 256, 0, st>>>(g_in, static_cast<double *>(G), count, scale);
+    else g_init_kernel<float><<<blocks, 256, 0, st>>>(g_in, static_cast<float *>(G), count, scale);
+    return cudaGetLastError();
+}
+
+// Eq. (5) keeps the [CLS] token (index 0) out of the transport problem: zero weight for it on both sides, uniform
+// weights over the other queries and over the other valid keys.
+__global__ void cls_marginals_kernel(float *__restrict__ a, float *__restrict__ b, const int32_t *key_len, int H, int nq,
+                                     int nk, int *status)
+{
+    const int bh = blockIdx.x, bb = bh / H;
+    int kv = nk;
+    if (key_len != nullptr) kv = min(max(key_len[bb], 0), nk);
+    if (threadIdx.x == 0 && (kv <= 1 || nq <= 1)) atomicOr(status, 2 /* LOT_DEV_EMPTY */);
+    const float wa = nq > 1 ? 1.f / (float)(nq - 1) : 0.f, wb = kv > 1 ? 1.f / (float)(kv - 1) : 0.f;
+    for (int i = threadIdx.x; i < nq; i += blockDim.x) a[(size_t)bh * nq + i] = i == 0 ? 0.f : wa;
+    for (int j = threadIdx.x; j < nk; j += blockDim.x) b[(size_t)bh * nk + j] = (j == 0 || j >= kv) ? 0.f : wb;
+}
+
+cudaError_t launch_cls_marginals(float *a, float *b, const int32_t *key_len, int B, int H, int nq, int nk, int *status,
+                                 cudaStream_t st)
+{
+    cls_marginals_kernel<<<B * H, 256, 0, st>>>(a, b, key_len, H, nq, nk, status);
+    return cudaGetLastError();
+}
+
+// One block per slice: scores tau <q_0, k_j> of the valid keys (kept in global scratch), their maximum, the
+// exponentials and their sum, then one thread per channel adds up the weighted values.
+template <typename T>
+__global__ void __launch_bounds__(256)
+cls_row_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, const int32_t *key_len, int H,
+               int nq, int nk, int d, float tau, float *__restrict__ scores, T *__restrict__ out)
+{
+    __shared__ float red[256];
+    __shared__ float q0[256];
+    const int bh = blockIdx.x, bb = bh / H;
+    int kv = nk;
+    if (key_len != nullptr) kv = min(max(key_len[bb], 0), nk);
+    const T *qb = q + (size_t)bh * nq * d, *kb = k + (size_t)bh * nk * d, *vb = v + (size_t)bh * nk * d;
+    float *sc = scores + (size_t)bh * nk;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) q0[c] = Elem<T>::load(qb + c);
+    __syncthreads();
+    float mx = neg_inf();
+    for (int j = threadIdx.x; j < kv; j += blockDim.x) {
+        float acc = 0.f;
+        for (int c = 0; c < d; c += 4) {
+            float kk[4];
+            load4(kb + (size_t)j * d + c, kk);
+            acc = fmaf(q0[c], kk[0], acc); acc = fmaf(q0[c + 1], kk[1], acc);
+            acc = fmaf(q0[c + 2], kk[2], acc); acc = fmaf(q0[c + 3], kk[3], acc);
+        }
+        acc *= tau;
+        sc[j] = acc;
+        mx = fmaxf(mx, acc);
+    }
+    red[threadIdx.x] = mx;
+    __syncthreads();
+    for (int off = 128; off > 0; off >>= 1) {
+        if (threadIdx.x < off) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + off]);
+        __syncthreads();
+    }
+    mx = red[0];
+    __syncthreads();
+    float den = 0.f;
+    for (int j = threadIdx.x; j < kv; j += blockDim.x) {
+        const float e = __expf(sc[j] - mx);
+        sc[j] = e;
+        den += e;
+    }
+    red[threadIdx.x] = den;
+    __syncthreads();
+    for (int off = 128; off > 0; off >>= 1) {
+        if (threadIdx.x < off) red[threadIdx.x] += red[threadIdx.x + off];
+        __syncthreads();
+    }
+    den = red[0];
+    __threadfence_block();
+    __syncthreads();
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        float acc = 0.f;
+        for (int j = 0; j < kv; ++j) acc = fmaf(sc[j], Elem<T>::load(vb + (size_t)j * d + c), acc);
+        Elem<T>::store(out + (size_t)bh * nq * d + c, kv > 0 ? acc / den : 0.f);
+    }
+}
+
+cudaError_t launch_cls_row(const void *q, const void *k, const void *v, const int32_t *key_len, int dtype, int B, int H,
+                           int nq, int nk, int d, float tau, float *scores, void *out, cudaStream_t st)
+{
+    if (dtype == 0)
+        cls_row_kernel<float><<<B * H, 256, 0, st>>>(static_cast<const float *>(q), static_cast<const float *>(k),
+                                                     static_cast<const float *>(v), key_len, H, nq, nk, d, tau, scores,
+                                                     static_cast<float *>(out));
+    else
+        cls_row_kernel<__nv_bfloat16><<<B * H, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(q),
+                                                             static_cast<const __nv_bfloat16 *>(k),
+                                                             static_cast<const __nv_bfloat16 *>(v), key_len, H, nq, nk, d, tau,
+                                                             scores, static_cast<__nv_bfloat16 *>(out));
     return cudaGetLastError();
 }
 
