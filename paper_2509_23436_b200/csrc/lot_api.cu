@@ -306,8 +306,8 @@ int lot_launch_count(int dtype, int B, int H, int n, int d, int r, int iters)
 {
     if (iters < 0) return 0;
     const int path = lot_path(dtype, B, H, n, d, r, iters);
-    if (path == kPathResident) return 1 + fused_launches(iters);    // the two streamed kernels return at once unless asked to redo
-    if (path == kPathStreamed) return fused_launches(iters);
+    if (path == kPathResident) return 1 + 2;                        // the two streamed kernels return at once unless asked to redo
+    if (path == kPathStreamed) return fused_launches(B, H, n, r, iters);
     return 2 + iters + 1 + 2;
 }
 

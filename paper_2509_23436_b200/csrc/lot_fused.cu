@@ -85,6 +85,9 @@ struct alignas(64) FusedParams {
     float *g1_out, *g2_out;      // [BH][r] final potentials, natural-log units, or nullptr
     const unsigned *redo;        // not nullptr: run only if *redo == redo_tag (a call that repeats a resident launch)
     unsigned redo_tag;
+    int ext_apply;               // 1: the apply stages run as separate kernels from the stored Gibbs kernel (lot_apply.cu);
+                                 // this kernel applies only the slices whose stored kernel cannot carry the final potentials
+    int *decision;               // [2][BH] per (side, slice), zero at the start: 1 = stored kernel good to the end, 2 = not
     int *status;
     int B, H, n, r, T;
     int TPS;                     // tiles per slice = ceil(n / 128)
@@ -198,8 +201,8 @@ struct Plan {
     static constexpr int offMisc = offBar + 64 * 8;            // abort flag, TMEM base, flags
     static constexpr int offG = offMisc + 128;                 // float sG[kGroups][64]
     static constexpr int offGc = offG + kGroups * 64 * 4;      // float sGc[kMaxLoc][64]: this CTA's copy of the potentials
-    static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust, sResFirst, sResLast [kMaxLoc]
-    static constexpr int offSeg = offState + 5 * kMaxLoc * 4;  // int sSeg[kMaxLoc][kSegInts]: static parts of the segments
+    static constexpr int offState = offGc + kMaxLoc * 64 * 4;  // int sDone, sIter, sRobust, sResFirst, sResLast, sDec [kMaxLoc]
+    static constexpr int offSeg = offState + 6 * kMaxLoc * 4;  // int sSeg[kMaxLoc][kSegInts]: static parts of the segments
     static constexpr int offWt = offSeg + kMaxLoc * kSegInts * 4; // float sWt[kMaxLoc][64]: weights 2^(G - max G) of the stored-kernel passes
     static constexpr int total = offWt + kMaxLoc * 64 * 4;
     // float sPart[2][kEpiWarps][64][2], the per-warp column pairs of the SUM passes, lives in the first plan buffer
@@ -382,6 +385,8 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     // attempt's answer.
     volatile int *sResFirst = sRobust + kMaxLoc;
     volatile int *sResLast = sResFirst + kMaxLoc;
+    // 1 = the stored kernel of this segment serves the apply kernels, 2 = it does not (written with the last pivot update)
+    volatile int *sDec = sResLast + kMaxLoc;
     volatile int *sPubDone = reinterpret_cast<volatile int *>(smem + PL::offMisc + 12);
     int *sSeg = reinterpret_cast<int *>(smem + PL::offSeg);
     // Wait until `need` attempts of local segment li (global index idx) are complete: 0 = gave up, else
@@ -409,6 +414,30 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BH = P.B * P.H;
+    // With the apply stages in their own kernels: does this kernel still apply slice g.s?  Only if the stored kernel of
+    // one of its sides cannot carry the final potentials.  A side of which this block holds tiles answers from shared
+    // memory once its last pivot update is in; the other side's answer is polled from global memory.  (One thread.)
+    // Returns 0 = gave up, 1 = skip the segment, 2 = apply it here.
+    auto apply_here = [&](const Seg &g, int s_lo) -> int {
+        if (!P.ext_apply) return 2;
+        int verdict = 1;
+        for (int side = 0; side < 2; ++side) {
+            const int li = (g.s - s_lo) * 2 + (side ? 0 : 1);
+            const int *e = sSeg + li * kSegInts;
+            int d;
+            if (e[5] < e[6]) {
+                if (!spin_ge(sIter + li, P.T, sAbort, P.status)) return 0;
+                d = sDec[li];
+            } else if (side == 1 && P.key_len != nullptr && __ldg(P.key_len + g.b) <= 0) {
+                d = 1;                      // no keys at all: nothing updates that side; the apply kernels write the zeros
+            } else {
+                if (!poll_ge(P.decision + side * BH + g.s, 1, sAbort, P.status)) return 0;
+                d = ld_acquire(P.decision + side * BH + g.s);
+            }
+            if (d == 2) verdict = 2;
+        }
+        return verdict;
+    };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(bar(bXFull + i), 1); mbar_init(bar(bXEmpty + i), 1); mbar_init(bar(bREmpty + i), 4); }
@@ -431,6 +460,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     for (int i = threadIdx.x; i < kMaxLoc * 64; i += kThreads) sGc[i] = 0.f;
     if (threadIdx.x < 3 * kMaxLoc) sDone[threadIdx.x] = 0;
     else if (threadIdx.x < 5 * kMaxLoc) sDone[threadIdx.x] = 0x7fffffff;
+    else if (threadIdx.x < 6 * kMaxLoc) sDone[threadIdx.x] = 0;
     if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxLoc) {
         // segment table: one thread per (slice, side) of this CTA
         const int li = threadIdx.x - 128;
@@ -486,6 +516,11 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     if (go == 0) { ok = false; break; }
                     if (g.extra && ((go - 1) & 1) == 0) continue;
                     resident = (go - 1) >> 1;
+                }
+                if (g.phase != kPhaseSum) {
+                    const int ah = apply_here(g, it.s_lo);
+                    if (ah == 0) { ok = false; break; }
+                    if (ah == 1) continue;
                 }
                 if (resident) {
                     // tiles of the stored Gibbs kernel instead of token tiles; no pivots, no MMA
@@ -620,6 +655,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     if (done == 0) { ok = false; break; }
                     continue;
                 }
+            }
+            if (g.phase != kPhaseSum) {
+                int ah = 0;
+                if (lane == 0) ah = apply_here(g, it.s_lo);
+                ah = __shfl_sync(0xffffffffu, ah, 0);
+                if (ah == 0) { ok = false; break; }
+                if (ah == 1) continue;
             }
             while (pend_k >= 0) issue_apply();
             if (w_open) {                                                    // W of the previous WRED segment complete
@@ -827,6 +869,18 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             for (int off = 16; off >= 1; off >>= 1) {
                 gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, off));
                 gmn = fminf(gmn, __shfl_xor_sync(0xffffffffu, gmn, off));
+            }
+            if (P.ext_apply && !fail && itn + 1 == P.T) {
+                // the last pivot update of this (slice, side): can the apply kernels work from its stored kernel?
+                const int dec = (RP == 64 && cached && !rb && P.Kt != nullptr && (gmx - gmn) <= 64.f) ? 1 : 2;
+                if (mine && g.slot == 0 && cached) {
+                    if (c0 < P.r) __stcg(P.G + (size_t)idx * RP + c0, sGc[li * 64 + c0]);
+                    if (c0 + 1 < P.r) __stcg(P.G + (size_t)idx * RP + c0 + 1, sGc[li * 64 + c0 + 1]);
+                }
+                if (lane == 0) {
+                    if (cached) sDec[li] = dec;
+                    if (g.slot == 0) { __threadfence(); st_release(P.decision + idx, dec); }
+                }
             }
             const bool run_started = cached && sResFirst[li] != 0x7fffffff, run_ended = cached && sResLast[li] != 0x7fffffff;
             const int next_resident = RP == 64 && cached && !fail && !rb && !run_ended && P.Kt != nullptr && (gmx - gmn) <= 64.f;
@@ -1164,6 +1218,13 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             const int idx = g.side * BH + g.s;
             // ---- WRED / OUT: wait until the final potential (and W') of this slice is known here
             const int li = g.li;
+            {
+                int ah = 0;
+                if (lane == 0) ah = apply_here(g, it.s_lo);
+                ah = __shfl_sync(0xffffffffu, ah, 0);
+                if (ah == 0) ok = false;
+                if (ah == 1) continue;
+            }
             if (gtid == 0) {
                 bool w = spin_ge(sPubDone, 1, sAbort, P.status);          // plan buffers free of SUM partials
                 if (w) w = li < kMaxLoc ? spin_ge(sIter + li, P.T, sAbort, P.status) : poll_ge(P.iter + idx, P.T, sAbort, P.status);
@@ -1464,6 +1525,22 @@ static inline int pad_r(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
 
 } // namespace fused
 
+// The apply stages run as separate kernels when the first pass keeps the Gibbs kernel (32 < r <= 64, more than one
+// iteration), every block caches the state of all its segments in shared memory, and the problem is large: measured on
+// B200 at B = 1, H = 16 the three-kernel form is 6 % faster at n = 65536, even at n = 16384 and 14 % slower at n = 4096
+// (two more launches), so it is taken from 4096 tiles per side on.
+bool fused_ext_apply(int B, int H, int n, int r, int iters)
+{
+    if (fused::pad_r(r) != 64 || iters < 2) return false;
+    if ((long long)B * H * ((n + 127) / 128) < 4096) return false;
+    int q, ctas, ms, cps;
+    fused_geometry(B, H, n, &q, &ctas, &ms, &cps);
+    if (cps > 0) return true;
+    const int TPS = (n + 127) / 128;
+    const int slices = (q + TPS - 2) / TPS + 1;           // most slices a block of q consecutive tiles can touch
+    return 2 * slices <= fused::kMaxLoc;
+}
+
 bool fused_supported(int dtype, int d, int r)
 {
     return dtype == 1 && d == fused::kDK && r >= 1 && r <= 64;
@@ -1507,11 +1584,13 @@ FusedLayout fused_layout(int B, int H, int n, int d, int r)
     L.robust = o; o += up256((size_t)2 * BH * 4);
     L.wflag = o; o += up256((size_t)BH * ms * 4);
     L.gnat = o; o += up256((size_t)2 * BH * r * 4);
+    L.decision = o; o += up256((size_t)2 * BH * 4);
     L.part = o; o += up256((size_t)2 * 2 * BH * ms * RP * 2 * 8);
     L.head_end = o;
     L.kt = o; o += RP == 64 ? up256((size_t)2 * BH * ((n + 127) / 128) * 128 * 64 * 2) : 0;
     L.zprep = o; o += up256((size_t)H * 2 * RP * d * 2);
     L.wpart = o; o += up256((size_t)BH * ms * 64 * d * 4);
+    L.wpart2 = o; o += fused_ext_apply(B, H, n, r, 2) ? up256(stored_apply_wpart_bytes(B, H, n)) : 0;
     L.total = o;
     return L;
 }
@@ -1571,6 +1650,8 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
     P.out = static_cast<__nv_bfloat16 *>(out);
     P.g1_out = g1_out; P.g2_out = g2_out;
     P.redo = redo; P.redo_tag = redo_tag;
+    P.ext_apply = fused_ext_apply(B, H, n, r, iters) && redo == nullptr ? 1 : 0;
+    P.decision = reinterpret_cast<int *>(w + L.decision);
     P.status = reinterpret_cast<int *>(w + L.status);
     P.B = B; P.H = H; P.n = n; P.r = r; P.T = iters;
     P.TPS = (n + 127) / 128;
@@ -1592,9 +1673,12 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
     if (RP == 16) e = launch_forward<16>(P, ctas, st);
     else if (RP == 32) e = launch_forward<32>(P, ctas, st);
     else e = launch_forward<64>(P, ctas, st);
-    return e;
+    if (e != cudaSuccess || !P.ext_apply) return e;
+    // the apply stages from the stored kernel, for every slice the Sinkhorn kernel left to them
+    return stored_apply(P.Kt, P.npad, P.G, beta, key_len, P.decision, v, out, reinterpret_cast<float *>(w + L.wpart2), P.status,
+                        B, H, n, r, st);
 }
 
-int fused_launches(int iters) { (void)iters; return 2; }
+int fused_launches(int B, int H, int n, int r, int iters) { return fused_ext_apply(B, H, n, r, iters) ? 4 : 2; }
 
 } // namespace lot

@@ -76,7 +76,7 @@ cudaError_t launch_cls_row(const void *q, const void *k, const void *v, const in
 
 // ---- fused tensor-core path (lot_fused.cu): bf16 tensors, d = 64, r <= 64 ----
 struct FusedLayout {
-    size_t status, G, epoch, iter, robust, wflag, gnat, head_end, kt, zprep, part, wpart, total;
+    size_t status, G, epoch, iter, robust, wflag, gnat, decision, head_end, kt, zprep, part, wpart, wpart2, total;
 };
 bool fused_supported(int dtype, int d, int r);
 void fused_geometry(int B, int H, int n, int *q, int *ctas, int *maxslots, int *cps);
@@ -86,7 +86,9 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
                             const int32_t *key_len, int B, int H, int n, int d, int r, float eps, int iters,
                             void *out, float *g1_out, float *g2_out, void *ws, const unsigned *redo, unsigned redo_tag,
                             cudaStream_t st);
-int fused_launches(int iters);
+int fused_launches(int B, int H, int n, int r, int iters);
+// true when the apply stages of a streamed call run as the two kernels of lot_apply.cu
+bool fused_ext_apply(int B, int H, int n, int r, int iters);
 
 // ---- resident tensor-core path (lot_resident.cu): bf16 tensors, d = 64, r <= 64, tiles fit one SM's TMEM + shared memory ----
 struct ResidentGeom {
@@ -102,6 +104,11 @@ ResidentLayout resident_layout(int B, int H, int n, int d, int r);
 cudaError_t resident_attention(const void *q, const void *k, const void *v, const float *z, const float *beta,
                                const int32_t *key_len, int B, int H, int n, int d, int r, float eps, int iters,
                                void *out, float *g1_out, float *g2_out, void *ws, unsigned *tag_out, cudaStream_t st);
-void resident_debug(int what, long long value);   // test hooks: 1 = block that skips its first publish (one call), 2 = wait limit in ns
+void resident_debug(int what, long long value);
+
+// ---- apply stages from the stored Gibbs kernel (lot_apply.cu), behind the streamed Sinkhorn kernel ----
+size_t stored_apply_wpart_bytes(int B, int H, int n);
+cudaError_t stored_apply(const void *kt, int npad, const float *G, const float *beta, const int32_t *key_len, const int *decision,
+                         const void *v, void *out, float *wpart, int *status, int B, int H, int n, int r, cudaStream_t st);   // test hooks: 1 = block that skips its first publish (one call), 2 = wait limit in ns
 
 } // namespace lot

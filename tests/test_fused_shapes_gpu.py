@@ -37,6 +37,9 @@ CASES = [
     (128, 12, 100, 64, 3, 0.1, False),
     (512, 3, 197, 16, 4, 0.1, True),
     (96, 4, 150, 64, 5, 0.01, False),
+    # 4096 tiles per side and more: the apply stages run as their own kernels, from the stored Gibbs kernel
+    (2, 16, 16384, 64, 3, 0.1, True),
+    (1, 33, 16384, 50, 2, 0.1, False),
     # the benchmark shapes of configs 2 and 3 at a training-size batch
     (64, 3, 197, 16, 10, 0.1, False),
     (32, 12, 512, 32, 20, 0.05, True),
