@@ -52,6 +52,8 @@ def parse():
     ap.add_argument("--dtype", default=None, choices=["bf16", "f32"])
     ap.add_argument("--shard", default="batch", choices=["batch", "heads"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--path", default="auto", choices=["auto", "general", "streamed", "resident"],
+                    help="kernel path the library takes where it can run (default: the library's own choice)")
     ap.add_argument("--iters", type=int, default=None,
                     help="Sinkhorn iterations (default: the configuration's); 0 = apply passes only")
     return ap.parse_args()
@@ -264,6 +266,8 @@ def run_ours(args):
     key_len = None if hkl is None else hkl.to(dev)
     out = torch.empty_like(q)
     code = lot.LOT_BF16 if q.dtype == torch.bfloat16 else lot.LOT_F32
+    if args.path != "auto":          # before the workspace is sized: its size follows the path
+        lot.lot_debug_hook(4, {"general": 0, "streamed": 1, "resident": 2}[args.path])
     ws = torch.empty(max(256, lot.lot_workspace_bytes(B, H, n, d, r, code)), device=dev, dtype=torch.uint8)
     flush = torch.empty(512 << 20, device=dev, dtype=torch.uint8)
     stream = torch.cuda.current_stream()

@@ -186,8 +186,8 @@ LOT_API int lot_launch_count(int dtype, int B, int H, int n, int d, int r, int i
  *   what = 3: device address of a trace buffer (8002 64-bit words, zeroed by the caller) into which thread block 0 of
  *             the resident path logs (event code, global timer) pairs, or 0 to stop; for profiling.
  *   what = 4: 1 or 2 makes lot_attention_fwd_ex take tensor-core path 1 or 2 of lot_path wherever that path can run
- *             at all (the default choice is by measured speed); -1 restores the default.  lot_path and
- *             lot_workspace_bytes follow the switch.
+ *             at all (the default choice is by measured speed), 0 the general path; -1 restores the default.
+ *             lot_path, lot_launch_count and lot_workspace_bytes follow the switch.
  * Returns LOT_ERR_INVALID_ARG for any other `what`.
  */
 LOT_API int lot_debug_hook(int what, long long value);
@@ -205,6 +205,29 @@ LOT_API int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
                          int dtype, int B, int H, int n, int d, int r, float eps, int iters,
                          void *out, float *g1_out, float *g2_out,
                          void *ws, size_t ws_bytes, lot_stream_t stream);
+
+/*
+ * lot_attention_bwd -- gradients of the forward path (Section "Learning": the pivots, their masses and the
+ * projections are trained by back-propagating through the two shared-eps Sinkhorn problems, Eq. (1)-(2), and the
+ * glued composition, Eq. (3)-(4)).  What is differentiated is exactly the map lot_attention_fwd_ex computes: the
+ * unrolled iteration (start at zero, `iters` times token update then pivot update, one closing token update),
+ * not the fixed point.  Given dout = d(loss)/d(out) it returns d(loss)/d(q, k, v, z, beta).
+ *   q,k,v,dout,dq,dk,dv [B,H,n,d] in `dtype` (device);  z, dz [H,r,d];  beta, dbeta [H,r] float32 (device);
+ *   key_len [B] int32 or NULL as in the forward (rows of dk, dv beyond the length are zero).
+ *   beta is treated as r free positive numbers per head (no simplex constraint: a softmax parametrisation is the
+ *   caller's chain rule); dz and dbeta are summed over the batch.
+ * The forward is recomputed (materialised similarities, general path arithmetic: float32 for bf16 tensors,
+ * float64 for float32 tensors); only the pivot potentials of every iteration are kept.  2*iters + 20 launches.
+ * ws: lot_bwd_workspace_bytes(...) bytes of device scratch, 256-byte aligned, owned by the caller; the device
+ * status word of the recomputed forward sits at its start (lot_device_status).
+ * Errors as lot_attention_fwd_ex.  B == 0 or n == 0: dz and dbeta are zero-filled, nothing else is touched.
+ */
+LOT_API size_t lot_bwd_workspace_bytes(int B, int H, int n, int d, int r, int dtype, int iters);
+LOT_API int lot_attention_bwd(const void *q, const void *k, const void *v, const float *z, const float *beta,
+                      const int32_t *key_len, const void *dout,
+                      int dtype, int B, int H, int n, int d, int r, float eps, int iters,
+                      void *dq, void *dk, void *dv, float *dz, float *dbeta,
+                      void *ws, size_t ws_bytes, lot_stream_t stream);
 
 /* Scratch bytes lot_attention_fwd_var needs for these sizes. */
 LOT_API size_t lot_var_workspace_bytes(int B, int H, int nq, int nk, int d, int r, int dtype);

@@ -39,6 +39,8 @@ SIGNATURES = {
     "lot_var_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "lot_attention_fwd_var": (_i, [_vp] * 10 + [_i, _f] + [_i] * 7 + [_f, _i] + [_vp, _vp, _vp, _vp, _sz, _vp]),
     "lot_attention_fwd": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp]),
+    "lot_bwd_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
+    "lot_attention_bwd": (_i, [_vp] * 7 + [_i] * 6 + [_f, _i] + [_vp] * 6 + [_sz, _vp]),
     "lot_device_status": (_i, [_vp, _vp, ctypes.POINTER(_i)]),
 }
 
@@ -238,3 +240,33 @@ def lot_device_status(ws: Optional[torch.Tensor], stream=None) -> int:
     st = lib().lot_device_status(_dev(ws, "ws"), _stream(stream), ctypes.byref(val))
     _check(st, "lot_device_status")
     return val.value
+
+
+def lot_bwd_workspace_bytes(B, H, n, d, r, dtype_code, iters) -> int:
+    return lib().lot_bwd_workspace_bytes(B, H, n, d, r, dtype_code, iters)
+
+
+def lot_attention_bwd(q, k, v, z, beta, key_len, dout, eps, iters, *, ws=None, stream=None):
+    """Gradients of the forward with respect to q, k, v, z, beta.  Returns (dq, dk, dv, dz, dbeta, ws)."""
+    B, H, n, d = q.shape
+    r = z.shape[1]
+    code = _dtype_code(q)
+    for name, t in (("k", k), ("v", v), ("dout", dout)):
+        if t.shape != q.shape or t.dtype != q.dtype:
+            raise LotError(f"{name} must have q's shape and dtype")
+    if tuple(z.shape) != (H, r, d) or tuple(beta.shape) != (H, r):
+        raise LotError("z must be [H,r,d] and beta [H,r]")
+    f32 = torch.float32
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    dz = torch.empty((H, r, d), device=q.device, dtype=f32)
+    dbeta = torch.empty((H, r), device=q.device, dtype=f32)
+    need = lot_bwd_workspace_bytes(B, H, n, d, r, code, int(iters))
+    if ws is None:
+        ws = torch.empty(max(need, 256), device=q.device, dtype=torch.uint8)
+    st = lib().lot_attention_bwd(_dev(q, "q"), _dev(k, "k"), _dev(v, "v"), _dev(z, "z", f32), _dev(beta, "beta", f32),
+                                 _dev(key_len, "key_len", torch.int32), _dev(dout, "dout", q.dtype),
+                                 code, B, H, n, d, r, float(eps), int(iters),
+                                 _dev(dq, "dq"), _dev(dk, "dk"), _dev(dv, "dv"), _dev(dz, "dz", f32),
+                                 _dev(dbeta, "dbeta", f32), _dev(ws, "ws"), ws.numel(), _stream(stream))
+    _check(st, "lot_attention_bwd")
+    return dq, dk, dv, dz, dbeta, ws

@@ -121,6 +121,47 @@ VarLayout var_layout(int B, int H, int nq, int nk, int d, int r, int dtype)
     return V;
 }
 
+// Workspace of lot_attention_bwd: the general path's blocks plus the kept potentials of every iteration, the
+// gradient with respect to the similarities and the small reduction buffers.
+struct BwdLayout {
+    size_t counter, counter2, hist, gamma, dbeta_acc, head_end, part, M, cost, dC, wpart, Wp, Xw, dWm, dbeta_direct, zt,
+        dzpart, total;
+    int chunks, rows_per_chunk, achunks, arows, dzchunks;
+};
+
+BwdLayout bwd_layout(int B, int H, int n, int d, int r, int dtype, int iters)
+{
+    BwdLayout L;
+    const size_t lt = dtype == LOT_F32 ? 8 : 4;
+    const int BH = B * H, np = 2 * BH;
+    const int tiles = ((r + 63) / 64) * ((d + 63) / 64) * BH;
+    L.chunks = pass_chunks(np > 0 ? np : 1, n > 0 ? n : 1);
+    L.rows_per_chunk = (n + L.chunks - 1) / L.chunks;
+    L.achunks = apply_chunks(BH > 0 ? BH : 1, n > 0 ? n : 1, r, d);
+    L.arows = (n + L.achunks - 1) / L.achunks;
+    L.dzchunks = bwd_dz_chunks(BH > 0 ? BH : 1, n > 0 ? n : 1, r, d);
+    size_t o = 256;                                   // status word at 0
+    L.counter = o; o += up256((size_t)np * 4);
+    L.counter2 = o; o += up256((size_t)tiles * 4);
+    L.hist = o; o += up256((size_t)(iters + 1) * np * r * lt);
+    L.gamma = o; o += up256((size_t)np * r * lt);
+    L.dbeta_acc = o; o += up256((size_t)np * r * lt);
+    L.head_end = o;
+    L.part = o; o += up256((size_t)np * L.chunks * r * 8);
+    L.M = o; o += up256((size_t)np * n * lt);
+    L.cost = o; o += up256((size_t)np * n * r * lt);
+    L.dC = o; o += up256((size_t)np * n * r * lt);
+    L.wpart = o; o += up256((size_t)BH * L.achunks * r * d * 4);
+    L.Wp = o; o += up256((size_t)BH * r * d * 4);
+    L.Xw = o; o += up256((size_t)BH * r * d * 4);
+    L.dWm = o; o += up256((size_t)BH * r * d * 4);
+    L.dbeta_direct = o; o += up256((size_t)BH * r * 4);
+    L.zt = o; o += up256((size_t)H * r * d * 4);
+    L.dzpart = o; o += up256((size_t)np * L.dzchunks * r * d * lt);
+    L.total = o;
+    return L;
+}
+
 template <typename T> inline T *at(void *ws, size_t off) { return reinterpret_cast<T *>(static_cast<char *>(ws) + off); }
 
 struct Managed {
@@ -147,12 +188,13 @@ void remember_ws(const void *ws, int path, unsigned tag, size_t fused_off)
 }
 
 enum { kPathGeneral = 0, kPathStreamed = 1, kPathResident = 2 };
-std::atomic<int> g_force_path{-1};      // test hook: 1 or 2 picks that tensor-core path wherever it can run
+std::atomic<int> g_force_path{-1};      // test hook: 0 picks the general path, 1 or 2 that tensor-core path wherever it can run
 int choose_path(int dtype, int B, int H, int n, int d, int r)
 {
     if (!fused_supported(dtype, d, r)) return kPathGeneral;
     const bool res_ok = B >= 1 && n >= 1 && resident_geometry(dtype, B, H, n, d, r).ok;
     const int force = g_force_path.load();
+    if (force == kPathGeneral) return kPathGeneral;
     if (force == kPathStreamed) return kPathStreamed;
     if (force == kPathResident) return res_ok ? kPathResident : kPathStreamed;
     // Measured on B200 (see the design notes): the resident kernel wins where the streamed one has no stored-kernel
@@ -462,7 +504,7 @@ int lot_attention_fwd_var(const void *q, const void *k, const void *v, const flo
     if (launch_cost(q, z, dtype, BH, H, nq, d, r, cost1, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
     if (launch_cost(k, z, dtype, BH, H, nk, d, r, cost2, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
 
-    PassArgs pa[2];
+    PassArgs pa[2] = {};
     for (int side = 0; side < 2; ++side) {
         const SinkLayout &L = side ? V.s2 : V.s1;
         PassArgs &x = pa[side];
@@ -562,6 +604,123 @@ int lot_device_status(const void *ws, lot_stream_t stream, int *status)
     const int mine = head[1] == rec.tag ? (int)head[0] : 0;
     // a call that was recomputed reports the recomputation's flags (and a timeout of the first attempt, if any)
     *status = head[2] == rec.tag ? (LOT_DEV_RECOMPUTED | streamed | (mine & LOT_DEV_TIMEOUT)) : (mine | streamed);
+    return LOT_OK;
+}
+
+size_t lot_bwd_workspace_bytes(int B, int H, int n, int d, int r, int dtype, int iters)
+{
+    if (dtype != LOT_F32 && dtype != LOT_BF16) return 0;
+    if (check_dims(B, H, n, r) != LOT_OK || check_d(n, d) != LOT_OK || iters < 0) return 0;
+    return bwd_layout(B, H, n, d, r, dtype, iters).total;
+}
+
+int lot_attention_bwd(const void *q, const void *k, const void *v, const float *z, const float *beta,
+                      const int32_t *key_len, const void *dout,
+                      int dtype, int B, int H, int n, int d, int r, float eps, int iters,
+                      void *dq, void *dk, void *dv, float *dz, float *dbeta,
+                      void *ws, size_t ws_bytes, lot_stream_t stream)
+{
+    if (dtype != LOT_F32 && dtype != LOT_BF16) return LOT_ERR_INVALID_ARG;
+    int st = check_dims(B, H, n, r);
+    if (st != LOT_OK) return st;
+    st = check_d(n, d);
+    if (st != LOT_OK) return st;
+    if (!(eps > 0.f) || !isfinite(eps) || iters < 0) return LOT_ERR_INVALID_ARG;
+    if (!z || !beta || !dz || !dbeta) return LOT_ERR_INVALID_ARG;
+    if (!aligned16(z) || !aligned16(beta) || !aligned16(dz) || !aligned16(dbeta)) return LOT_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (B == 0 || n == 0) {
+        // no tokens: the pivots receive no gradient
+        if (cudaMemsetAsync(dz, 0, (size_t)H * r * d * sizeof(float), s) != cudaSuccess) return LOT_ERR_CUDA;
+        if (cudaMemsetAsync(dbeta, 0, (size_t)H * r * sizeof(float), s) != cudaSuccess) return LOT_ERR_CUDA;
+        return LOT_OK;
+    }
+    if (!q || !k || !v || !dout || !dq || !dk || !dv) return LOT_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) || !aligned16(dk) ||
+        !aligned16(dv) || (key_len && (reinterpret_cast<uintptr_t>(key_len) & 3u)))
+        return LOT_ERR_INVALID_ARG;
+    const BwdLayout L = bwd_layout(B, H, n, d, r, dtype, iters);
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < L.total) return LOT_ERR_WORKSPACE;
+    remember_ws(ws, kPathGeneral, 0, 0);
+    const bool wide = dtype == LOT_F32;
+    const size_t lt = wide ? 8 : 4;
+    const int BH = B * H, np = 2 * BH;
+    const int ttype = dtype == LOT_F32 ? 0 : 1;        // tensor element type for the products
+    const int ltype = wide ? 2 : 0;                    // type of the similarity-sized buffers
+    if (cudaMemsetAsync(ws, 0, L.head_end, s) != cudaSuccess) return LOT_ERR_CUDA;
+
+    // ---- the forward, keeping the potentials of every iteration
+    char *cost1 = at<char>(ws, L.cost);
+    char *cost2 = cost1 + (size_t)BH * n * r * lt;
+    if (launch_cost(q, z, dtype, BH, H, n, d, r, cost1, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_cost(k, z, dtype, BH, H, n, d, r, cost2, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    char *hist = at<char>(ws, L.hist);
+    const size_t hstep = (size_t)np * r * lt;
+    PassArgs a{};
+    a.cost = cost1; a.beta = beta; a.len = key_len; a.len_from = BH;
+    a.part = at<float>(ws, L.part); a.counter = at<unsigned>(ws, L.counter);
+    a.M = at<void>(ws, L.M); a.status = at<int>(ws, 0);
+    a.nprob = np; a.B = B; a.H = H; a.n = n; a.r = r;
+    a.chunks = L.chunks; a.rows_per_chunk = L.rows_per_chunk;
+    a.mode = wide ? kModeWide : kModeF32;
+    a.scale_d = 1.4426950408889634 / (double)eps;
+    a.eps_ln2 = (float)((double)eps * 0.6931471805599453);
+    for (int it = 0; it < iters; ++it) {
+        a.G = hist + (size_t)it * hstep; a.G_next = hist + (size_t)(it + 1) * hstep;
+        if (launch_sinkhorn_pass(a, false, s) != cudaSuccess) return LOT_ERR_CUDA;
+    }
+    char *Gfin = hist + (size_t)iters * hstep;
+    a.G = Gfin; a.G_next = nullptr;
+    if (launch_sinkhorn_pass(a, true, s) != cudaSuccess) return LOT_ERR_CUDA;
+
+    char *M1 = at<char>(ws, L.M), *M2 = M1 + (size_t)BH * n * lt;
+    char *G1 = Gfin, *G2 = Gfin + (size_t)BH * r * lt;
+    float *Wp = at<float>(ws, L.Wp), *Xw = at<float>(ws, L.Xw), *dWm = at<float>(ws, L.dWm);
+    ApplyArgs ap{};
+    ap.cost1 = cost1; ap.cost2 = cost2; ap.G1 = G1; ap.G2 = G2; ap.M1 = M1; ap.M2 = M2;
+    ap.beta = beta; ap.key_len = key_len; ap.v = v; ap.out = nullptr;
+    ap.wpart = at<float>(ws, L.wpart); ap.Wp = Wp; ap.counter = at<unsigned>(ws, L.counter2);
+    ap.B = B; ap.H = H; ap.n = n; ap.nk = n; ap.d = d; ap.r = r;
+    ap.chunks = L.achunks; ap.rows_per_chunk = L.arows; ap.scale_d = a.scale_d;
+    if (launch_apply_w(ap, dtype, s) != cudaSuccess) return LOT_ERR_CUDA;                 // W' = Diag(1/beta) Gamma2 V
+
+    // ---- reverse of the read-out, Eq. (4): out = R1 W'
+    ApplyArgs aq = ap;                                  // R1^T dout / (n beta): the key-side kernel on the query side
+    aq.cost2 = cost1; aq.G2 = G1; aq.M2 = M1; aq.key_len = nullptr; aq.v = dout; aq.Wp = Xw;
+    if (launch_apply_w(aq, dtype, s) != cudaSuccess) return LOT_ERR_CUDA;
+    float *dbd = at<float>(ws, L.dbeta_direct);
+    if (launch_bwd_w_fix(Xw, Wp, key_len, dWm, dbd, B, H, n, d, r, s) != cudaSuccess) return LOT_ERR_CUDA;
+    ApplyArgs av = ap;                                  // dV = Gamma2 dW: the query-side kernel on the key side
+    av.cost1 = cost2; av.G1 = G2; av.M1 = M2; av.Wp = dWm; av.out = dv;
+    if (launch_apply_out(av, dtype, s) != cudaSuccess) return LOT_ERR_CUDA;
+    char *dC1 = at<char>(ws, L.dC);
+    char *dC2 = dC1 + (size_t)BH * n * r * lt;
+    if (launch_gemm_nt(dout, ttype, Wp, false, dC1, ltype, BH, H, n, d, r, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_gemm_nt(v, ttype, dWm, false, dC2, ltype, BH, H, n, d, r, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+
+    // ---- reverse of the closing token update, then of the iterations, last first
+    BwdRowArgs br{};
+    br.cost = cost1; br.dC = dC1; br.gamma = at<void>(ws, L.gamma); br.dbeta_acc = at<void>(ws, L.dbeta_acc);
+    br.beta = beta; br.len = key_len; br.len_from = BH;
+    br.part = at<void>(ws, L.part); br.counter = at<unsigned>(ws, L.counter);
+    br.nprob = np; br.B = B; br.H = H; br.n = n; br.r = r;
+    br.chunks = L.chunks; br.rows_per_chunk = L.rows_per_chunk;
+    br.scale_d = a.scale_d; br.eps = (double)eps;
+    br.Ga = Gfin; br.Gb = nullptr;
+    if (launch_bwd_rows(br, true, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    for (int it = iters; it >= 1; --it) {
+        br.Ga = hist + (size_t)(it - 1) * hstep; br.Gb = hist + (size_t)it * hstep;
+        if (launch_bwd_rows(br, false, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    }
+
+    // ---- C = X Z^T: dX = dC Z, dZ = dC^T X
+    float *zt = at<float>(ws, L.zt);
+    if (launch_transpose_z(z, zt, H, r, d, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_gemm_nt(dC1, ltype, zt, true, dq, ttype, BH, H, n, r, d, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_gemm_nt(dC2, ltype, zt, true, dk, ttype, BH, H, n, r, d, wide, s) != cudaSuccess) return LOT_ERR_CUDA;
+    if (launch_bwd_dz(dC1, q, k, dtype, at<void>(ws, L.dzpart), dbd, br.dbeta_acc, dz, dbeta, B, H, n, d, r, L.dzchunks, wide,
+                      s) != cudaSuccess)
+        return LOT_ERR_CUDA;
     return LOT_OK;
 }
 

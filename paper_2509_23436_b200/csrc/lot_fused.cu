@@ -359,7 +359,9 @@ __device__ __forceinline__ void tmem_ld_quad(uint32_t taddr, float *v)
 // ---------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------
-template <int RP>
+// EXT: the variant whose apply stages may be left to the kernels of lot_apply.cu (P.ext_apply); the plain variant
+// carries none of that code.
+template <int RP, bool EXT>
 __global__ void __launch_bounds__(kThreads, 1)
 fused_forward_kernel(const __grid_constant__ FusedParams P)
 {
@@ -419,7 +421,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
     // memory once its last pivot update is in; the other side's answer is polled from global memory.  (One thread.)
     // Returns 0 = gave up, 1 = skip the segment, 2 = apply it here.
     auto apply_here = [&](const Seg &g, int s_lo) -> int {
-        if (!P.ext_apply) return 2;
+        if (!EXT || !P.ext_apply) return 2;
         int verdict = 1;
         for (int side = 0; side < 2; ++side) {
             const int li = (g.s - s_lo) * 2 + (side ? 0 : 1);
@@ -517,7 +519,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     if (g.extra && ((go - 1) & 1) == 0) continue;
                     resident = (go - 1) >> 1;
                 }
-                if (g.phase != kPhaseSum) {
+                if (EXT && g.phase != kPhaseSum) {
                     const int ah = apply_here(g, it.s_lo);
                     if (ah == 0) { ok = false; break; }
                     if (ah == 1) continue;
@@ -656,7 +658,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                     continue;
                 }
             }
-            if (g.phase != kPhaseSum) {
+            if (EXT && g.phase != kPhaseSum) {
                 int ah = 0;
                 if (lane == 0) ah = apply_here(g, it.s_lo);
                 ah = __shfl_sync(0xffffffffu, ah, 0);
@@ -870,7 +872,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
                 gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, off));
                 gmn = fminf(gmn, __shfl_xor_sync(0xffffffffu, gmn, off));
             }
-            if (P.ext_apply && !fail && itn + 1 == P.T) {
+            if (EXT && P.ext_apply && !fail && itn + 1 == P.T) {
                 // the last pivot update of this (slice, side): can the apply kernels work from its stored kernel?
                 const int dec = (RP == 64 && cached && !rb && P.Kt != nullptr && (gmx - gmn) <= 64.f) ? 1 : 2;
                 if (mine && g.slot == 0 && cached) {
@@ -1218,7 +1220,7 @@ fused_forward_kernel(const __grid_constant__ FusedParams P)
             const int idx = g.side * BH + g.s;
             // ---- WRED / OUT: wait until the final potential (and W') of this slice is known here
             const int li = g.li;
-            {
+            if (EXT) {
                 int ah = 0;
                 if (lane == 0) ah = apply_here(g, it.s_lo);
                 ah = __shfl_sync(0xffffffffu, ah, 0);
@@ -1595,13 +1597,13 @@ FusedLayout fused_layout(int B, int H, int n, int d, int r)
     return L;
 }
 
-template <int RP>
+template <int RP, bool EXT>
 static cudaError_t launch_forward(const fused::FusedParams &P, int ctas, cudaStream_t st)
 {
     // the attribute is per device: remember where it has been set
     static std::mutex mu;
     static bool attr_set[64] = {};
-    auto kern = fused::fused_forward_kernel<RP>;
+    auto kern = fused::fused_forward_kernel<RP, EXT>;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     {
@@ -1670,9 +1672,10 @@ cudaError_t fused_attention(const void *q, const void *k, const void *v, const f
                                          B, H, r, RP, d, scale, g1_out, g2_out, iters, redo, redo_tag);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-    if (RP == 16) e = launch_forward<16>(P, ctas, st);
-    else if (RP == 32) e = launch_forward<32>(P, ctas, st);
-    else e = launch_forward<64>(P, ctas, st);
+    if (RP == 16) e = launch_forward<16, false>(P, ctas, st);
+    else if (RP == 32) e = launch_forward<32, false>(P, ctas, st);
+    else if (P.ext_apply) e = launch_forward<64, true>(P, ctas, st);
+    else e = launch_forward<64, false>(P, ctas, st);
     if (e != cudaSuccess || !P.ext_apply) return e;
     // the apply stages from the stored kernel, for every slice the Sinkhorn kernel left to them
     return stored_apply(P.Kt, P.npad, P.G, beta, key_len, P.decision, v, out, reinterpret_cast<float *>(w + L.wpart2), P.status,

@@ -24,6 +24,7 @@ struct PassArgs {
     const float *mass;   // [nprob][n] token weights (>= 0; zero takes the token out of the problem), or nullptr:
                          // uniform over the valid tokens
     void *G;             // [nprob][r] pivot potentials, base-2 log units (in/out; float or double)
+    void *G_next;        // not nullptr: the updated potentials go here and G stays as it was (a kept history)
     float *part;         // [nprob][chunks][r][2] per-block column pairs (kappa, S)
     unsigned *counter;   // [nprob] arrival tickets, zero on entry and on exit
     void *M;             // final pass: [nprob][n] row log-sum-exp (base 2), +inf for massless rows
@@ -73,6 +74,46 @@ cudaError_t launch_cls_marginals(float *a, float *b, const int32_t *key_len, int
 // row 0 of every slice: softmax_j(tau <q_0, k_j>) over the valid keys, applied to v; scores: [BH][nk] scratch
 cudaError_t launch_cls_row(const void *q, const void *k, const void *v, const int32_t *key_len, int dtype, int B, int H,
                            int nq, int nk, int d, float tau, float *scores, void *out, cudaStream_t st);
+
+// ---- backward of the general path (lot_backward.cu) ----
+// One reverse step over a set of Sinkhorn problems (same problem numbering as PassArgs).  close: the closing token
+// update and the plan read-out; otherwise one (token update, pivot update) pair of the unrolled iteration.
+struct BwdRowArgs {
+    const void *cost;    // [nprob][n][r] similarities (float or double per `wide`)
+    void *dC;            // [nprob][n][r] same type.  close: in = gradient with respect to the row-stochastic plan,
+                         // out = gradient with respect to the similarities; otherwise updated in place
+    const void *Ga;      // [nprob][r] potentials the rows are normalised with (base-2 units)
+    const void *Gb;      // [nprob][r] potentials after the pivot update being reversed (not close)
+    void *gamma;         // [nprob][r] gradient with respect to the potentials in natural units: written by close,
+                         // read and replaced otherwise
+    void *dbeta_acc;     // [nprob][r] accumulates eps * gamma / beta over the reversed pivot updates
+    const float *beta;   // [H][r]
+    const int32_t *len;  // [B] or nullptr
+    int len_from;
+    void *part;          // [nprob][chunks][r] per-block column sums
+    unsigned *counter;   // [nprob] arrival tickets, zero on entry and on exit
+    int nprob, B, H, n, r;
+    int chunks, rows_per_chunk;
+    double scale_d;      // log2(e)/eps
+    double eps;
+};
+cudaError_t launch_bwd_rows(const BwdRowArgs &a, bool close, bool wide, cudaStream_t st);
+// out[s][i][j] = sum_k A[s][i][k] * Bm[(per_head ? s % H : s)][j][k]   (A: n x K, Bm: J x K, out: n x J)
+// a_type / out_type: 0 float, 1 bf16, 2 double; Bm is float
+cudaError_t launch_gemm_nt(const void *A, int a_type, const float *Bm, bool per_head, void *out, int out_type,
+                           int S, int H, int n, int K, int J, bool acc_double, cudaStream_t st);
+// Xw = (apply_w output of the query side on dout) -> dWm = Xw * n / nvalid_b (zero without keys),
+// dbeta_direct[s][t] = -n * sum_c Xw[s][t][c] * Wp[s][t][c]
+cudaError_t launch_bwd_w_fix(const float *Xw, const float *Wp, const int32_t *key_len, float *dWm, float *dbeta_direct,
+                             int B, int H, int n, int d, int r, cudaStream_t st);
+// zt[h][c][t] = z[h][t][c]
+cudaError_t launch_transpose_z(const float *z, float *zt, int H, int r, int d, cudaStream_t st);
+int bwd_dz_chunks(int BH, int n, int r, int d);
+// dz[h][t][c] = sum over b, side, rows of dC[side][b,h][i][t] * x_side[b,h][i][c];  dbeta[h][t] = sum over b of
+// dbeta_direct + both sides' dbeta_acc.  part: [2*BH][chunks][r][d] floats or doubles per `wide`
+cudaError_t launch_bwd_dz(const void *dC, const void *q, const void *k, int dtype, void *part, const float *dbeta_direct,
+                          const void *dbeta_acc, float *dz, float *dbeta, int B, int H, int n, int d, int r, int chunks,
+                          bool wide, cudaStream_t st);
 
 // ---- fused tensor-core path (lot_fused.cu): bf16 tensors, d = 64, r <= 64 ----
 struct FusedLayout {

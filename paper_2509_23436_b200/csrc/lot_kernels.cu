@@ -91,31 +91,66 @@ cudaError_t launch_cost(const void *x, const float *z, int dtype, int BH, int H,
 // One Sinkhorn pass (Eq. (1)-(2), scaling form).  With the token potential eliminated,
 //   token update : M_i = log2 sum_t 2^(L_it + G_t)                       (row log-sum-exp)
 //   pivot update : G_t += log2(beta_t / m) - log2 sum_i 2^(L_it + G_t - M_i)
-// where m = 1/n_valid is the token mass.  Rows are spread over GS lanes (GS = 8, 16 or
-// 32), each lane holding CPL columns t = lane + k*GS; row reductions are shuffles, column
-// sums are carried per lane as (kappa, S) pairs and merged lane -> warp -> block -> grid.
+// where m = 1/n_valid is the token mass.  A row is spread over LPR adjacent lanes (4, 8 or
+// 16); a lane holds NV groups of four adjacent columns, group v of lane c being columns
+// 4*(v*LPR + c) .. +3, so that the lanes of a warp read consecutive 16-byte pieces of
+// consecutive rows.  kRowsPerThread rows are in flight per thread.  Row reductions are
+// shuffles inside the LPR lanes; column sums are carried per lane as (kappa, S) pairs and
+// merged lane -> warp -> block -> grid in a fixed order.
 // FINAL = closing token update: writes M (and optionally g, f, plan), no pivot update.
 // ------------------------------------------------------------------------------------
 constexpr int kPassWarps = 8;
+constexpr int kRowsPerThread = 2;
+
+template <typename CostT>
+__device__ __forceinline__ void load_cost4(const CostT *p, bool vec, int t, int r, CostT (&c)[4]);
+
+template <>
+__device__ __forceinline__ void load_cost4<float>(const float *p, bool vec, int t, int r, float (&c)[4])
+{
+    if (vec) {
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(p));
+        c[0] = v.x; c[1] = v.y; c[2] = v.z; c[3] = v.w;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) c[j] = t + j < r ? __ldg(p + j) : 0.f;
+    }
+}
+
+template <>
+__device__ __forceinline__ void load_cost4<double>(const double *p, bool vec, int t, int r, double (&c)[4])
+{
+    if (vec) {
+        const double2 v0 = __ldg(reinterpret_cast<const double2 *>(p));
+        const double2 v1 = __ldg(reinterpret_cast<const double2 *>(p) + 1);
+        c[0] = v0.x; c[1] = v0.y; c[2] = v1.x; c[3] = v1.y;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) c[j] = t + j < r ? __ldg(p + j) : 0.0;
+    }
+}
 
 // CostT = stored similarity type, LT = type the logits, potentials and row LSE are assembled
 // in (float for bf16 tensors; double when the caller's tensors are float32, so that logits of
 // magnitude ~1e3 at small eps keep an absolute accuracy well below the 1e-4 output tolerance).
-template <int GS, int CPL, bool FINAL, typename CostT, typename LT>
+template <int LPR, int NV, bool FINAL, typename CostT, typename LT>
 __global__ void __launch_bounds__(kPassWarps * 32)
 sinkhorn_pass_kernel(PassArgs a)
 {
     __shared__ float sm_k[kPassWarps][256];
     __shared__ float sm_s[kPassWarps][256];
     __shared__ int sm_last;
+    constexpr int CPL = 4 * NV;
+    constexpr int RPW = 32 / LPR;                    // rows per warp and step
+    constexpr int RT = kRowsPerThread;
     const int p = blockIdx.x / a.chunks, chunk = blockIdx.x % a.chunks;
     const int slice = p % (a.B * a.H), b = slice / a.H, h = slice % a.H;
     int nvalid = a.n;
     if (a.len != nullptr && p >= a.len_from) nvalid = min(max(a.len[b], 0), a.n);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    constexpr int RPW = 32 / GS;
-    const int sub = lane / GS, cl = lane % GS;
+    const int sub = lane / LPR, cl = lane % LPR;
     const int r = a.r;
+    const bool vec = (r & 3) == 0;                   // rows start on 16-byte boundaries
     const CostT *C = static_cast<const CostT *>(a.cost) + (size_t)p * a.n * r;
     LT *Gp = static_cast<LT *>(a.G) + (size_t)p * r;
     LT *Mp = static_cast<LT *>(a.M) + (size_t)p * a.n;
@@ -124,12 +159,10 @@ sinkhorn_pass_kernel(PassArgs a)
 
     LT Gk[CPL];
     float kap[CPL], S[CPL];
-    bool cv[CPL];
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
-        int t = cl + k * GS;
-        cv[k] = t < r;
-        Gk[k] = cv[k] ? Gp[t] : (LT)0;
+        const int t = ((k >> 2) * LPR + cl) * 4 + (k & 3);
+        Gk[k] = t < r ? Gp[t] : (LT)neg_inf();        // columns beyond r: logit -inf, term 0
         kap[k] = neg_inf();
         S[k] = 0.f;
     }
@@ -140,48 +173,68 @@ sinkhorn_pass_kernel(PassArgs a)
     const float log2m = -lg2((float)max(nvalid, 1));
     const float mass = 1.f / (float)max(nvalid, 1);
 
-    for (int base = row0 + warp * RPW; base < loop_end; base += kPassWarps * RPW) {
-        const int i = base + sub;
-        const float mi = (mass_p != nullptr && i < row1) ? __ldg(mass_p + i) : mass;
-        const bool rv = i < row1 && mi > 0.f;
-        const float lmi = mass_p != nullptr ? lg2(mi) : log2m;      // log2 of this token's weight
-        LT l[CPL];
-        LT m = (LT)neg_inf();
+    for (int base = row0 + warp * (RPW * RT); base < loop_end; base += kPassWarps * RPW * RT) {
+        CostT c[RT][CPL];
+        float mi[RT];
+        bool rv[RT];
 #pragma unroll
-        for (int k = 0; k < CPL; ++k) {
-            LT c = (rv && cv[k]) ? (LT)__ldg(C + (size_t)i * r + cl + k * GS) : (LT)0;
-            l[k] = cv[k] ? fma(c, scale, Gk[k]) : (LT)neg_inf();
-            m = fmax(m, l[k]);
+        for (int u = 0; u < RT; ++u) {
+            const int i = base + u * RPW + sub;
+            mi[u] = (mass_p != nullptr && i < row1) ? __ldg(mass_p + i) : mass;
+            rv[u] = i < row1 && mi[u] > 0.f;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int t = (v * LPR + cl) * 4;
+                CostT cc[4] = {(CostT)0, (CostT)0, (CostT)0, (CostT)0};
+                if (rv[u] && t < r) load_cost4<CostT>(C + (size_t)i * r + t, vec, t, r, cc);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) c[u][v * 4 + j] = cc[j];
+            }
         }
 #pragma unroll
-        for (int off = GS / 2; off > 0; off >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, off));
-        float e[CPL];
-        float s = 0.f;
+        for (int u = 0; u < RT; ++u) {
+            const int i = base + u * RPW + sub;
+            const float lmi = mass_p != nullptr ? lg2(mi[u]) : log2m;      // log2 of this token's weight
+            LT l[CPL];
+            LT m = (LT)neg_inf();
 #pragma unroll
-        for (int k = 0; k < CPL; ++k) {
-            e[k] = (float)(l[k] - m);          // <= 0, exact difference of nearby logits
-            s += ex2(e[k]);
-        }
-#pragma unroll
-        for (int off = GS / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-        const float lgs = lg2(s);
-        if (!FINAL) {
-            if (rv) {
-#pragma unroll
-                for (int k = 0; k < CPL; ++k)
-                    if (cv[k]) pair_add(kap[k], S[k], mass_p != nullptr ? e[k] - lgs + lmi : e[k] - lgs);
+            for (int k = 0; k < CPL; ++k) {
+                l[k] = fma((LT)c[u][k], scale, Gk[k]);
+                m = fmax(m, l[k]);
             }
-        } else if (i < row_end) {
-            if (cl == 0) {
-                const LT Mi = m + (LT)lgs;
-                Mp[i] = rv ? Mi : (LT)__int_as_float(0x7f800000);
-                if (a.f_out) a.f_out[(size_t)p * a.n + i] = rv ? (float)((LT)a.eps_ln2 * ((LT)lmi - Mi)) : neg_inf();
-            }
-            if (a.plan_out) {
 #pragma unroll
-                for (int k = 0; k < CPL; ++k)
-                    if (cv[k])
-                        a.plan_out[((size_t)p * a.n + i) * r + cl + k * GS] = rv ? mi * ex2(e[k] - lgs) : 0.f;
+            for (int off = LPR / 2; off > 0; off >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, off));
+            float e[CPL];
+            float s = 0.f;
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) {
+                e[k] = (float)(l[k] - m);          // <= 0, exact difference of nearby logits
+                s += ex2(e[k]);
+            }
+#pragma unroll
+            for (int off = LPR / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+            const float lgs = lg2(s);
+            if (!FINAL) {
+                if (rv[u]) {
+                    const float shift = mass_p != nullptr ? lmi - lgs : -lgs;
+#pragma unroll
+                    for (int k = 0; k < CPL; ++k)
+                        if (e[k] > neg_inf()) pair_add(kap[k], S[k], e[k] + shift);
+                }
+            } else if (i < row_end) {
+                if (cl == 0) {
+                    const LT Mi = m + (LT)lgs;
+                    Mp[i] = rv[u] ? Mi : (LT)__int_as_float(0x7f800000);
+                    if (a.f_out)
+                        a.f_out[(size_t)p * a.n + i] = rv[u] ? (float)((LT)a.eps_ln2 * ((LT)lmi - Mi)) : neg_inf();
+                }
+                if (a.plan_out) {
+#pragma unroll
+                    for (int k = 0; k < CPL; ++k) {
+                        const int t = ((k >> 2) * LPR + cl) * 4 + (k & 3);
+                        if (t < r) a.plan_out[((size_t)p * a.n + i) * r + t] = rv[u] ? mi[u] * ex2(e[k] - lgs) : 0.f;
+                    }
+                }
             }
         }
     }
@@ -193,7 +246,7 @@ sinkhorn_pass_kernel(PassArgs a)
 
     // lanes of different row groups hold the same columns: merge them, then the warps
 #pragma unroll
-    for (int off = GS; off < 32; off <<= 1) {
+    for (int off = LPR; off < 32; off <<= 1) {
 #pragma unroll
         for (int k = 0; k < CPL; ++k) {
             float k2 = __shfl_xor_sync(0xffffffffu, kap[k], off);
@@ -203,11 +256,13 @@ sinkhorn_pass_kernel(PassArgs a)
     }
     if (sub == 0) {
 #pragma unroll
-        for (int k = 0; k < CPL; ++k)
-            if (cv[k]) {
-                sm_k[warp][cl + k * GS] = kap[k];
-                sm_s[warp][cl + k * GS] = S[k];
+        for (int k = 0; k < CPL; ++k) {
+            const int t = ((k >> 2) * LPR + cl) * 4 + (k & 3);
+            if (t < r) {
+                sm_k[warp][t] = kap[k];
+                sm_s[warp][t] = S[k];
             }
+        }
     }
     __syncthreads();
     const int t = threadIdx.x;
@@ -241,7 +296,7 @@ sinkhorn_pass_kernel(PassArgs a)
             // uniform weights: the common factor 1/nvalid was left out of the column sums
             LT gn = Gp[t] + (LT)lg2(a.mass ? a.beta[h * r + t] : a.beta[h * r + t] * (float)nvalid) - lam;
             if (!isfinite((float)gn)) atomicOr(a.status, 1 /* LOT_DEV_NONFINITE */);
-            Gp[t] = gn;
+            (a.G_next != nullptr ? static_cast<LT *>(a.G_next) + (size_t)p * r : Gp)[t] = gn;
         }
     }
     if (threadIdx.x == 0) a.counter[p] = 0u;
@@ -256,14 +311,14 @@ int pass_chunks(int nprob, int n)
     return c < 1 ? 1 : c;
 }
 
-template <int GS, int CPL, typename CostT, typename LT>
+template <int LPR, int NV, typename CostT, typename LT>
 static cudaError_t launch_pass_t(const PassArgs &a, bool final_pass, cudaStream_t st)
 {
     dim3 grid((unsigned)(a.nprob * a.chunks));
     if (final_pass)
-        sinkhorn_pass_kernel<GS, CPL, true, CostT, LT><<<grid, kPassWarps * 32, 0, st>>>(a);
+        sinkhorn_pass_kernel<LPR, NV, true, CostT, LT><<<grid, kPassWarps * 32, 0, st>>>(a);
     else
-        sinkhorn_pass_kernel<GS, CPL, false, CostT, LT><<<grid, kPassWarps * 32, 0, st>>>(a);
+        sinkhorn_pass_kernel<LPR, NV, false, CostT, LT><<<grid, kPassWarps * 32, 0, st>>>(a);
     return cudaGetLastError();
 }
 
@@ -271,12 +326,11 @@ template <typename CostT, typename LT>
 static cudaError_t launch_pass_r(const PassArgs &a, bool final_pass, cudaStream_t st)
 {
     const int r = a.r;
-    if (r <= 8) return launch_pass_t<8, 1, CostT, LT>(a, final_pass, st);
-    if (r <= 16) return launch_pass_t<16, 1, CostT, LT>(a, final_pass, st);
-    if (r <= 32) return launch_pass_t<32, 1, CostT, LT>(a, final_pass, st);
-    if (r <= 64) return launch_pass_t<32, 2, CostT, LT>(a, final_pass, st);
-    if (r <= 128) return launch_pass_t<32, 4, CostT, LT>(a, final_pass, st);
-    return launch_pass_t<32, 8, CostT, LT>(a, final_pass, st);
+    if (r <= 16) return launch_pass_t<4, 1, CostT, LT>(a, final_pass, st);
+    if (r <= 32) return launch_pass_t<4, 2, CostT, LT>(a, final_pass, st);
+    if (r <= 64) return launch_pass_t<4, 4, CostT, LT>(a, final_pass, st);
+    if (r <= 128) return launch_pass_t<8, 4, CostT, LT>(a, final_pass, st);
+    return launch_pass_t<16, 4, CostT, LT>(a, final_pass, st);
 }
 
 cudaError_t launch_sinkhorn_pass(const PassArgs &a, bool final_pass, cudaStream_t st)

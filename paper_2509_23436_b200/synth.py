@@ -106,3 +106,10 @@ def config(cfg: int, *, dtype=None, n=None, r=None, iters=None, eps=None, B=None
                     eps=eps or 0.1, iters=20 if iters is None else iters, qk="mixture",
                     name=f"cfg5-stress-r{r or 64}")
     raise ValueError(cfg)
+
+
+def cotangent(x: "LotInputs", seed: int = 1):
+    """A seeded upstream gradient for the backward tests: N(0,1) of out's shape, rounded to the tensor dtype."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(int(x.meta["seed"]) * 7919 + int(seed))
+    return torch.randn(x.q.shape, generator=gen, dtype=torch.float32).to(x.q.dtype).contiguous()
