@@ -54,6 +54,8 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--path", default="auto", choices=["auto", "general", "streamed", "resident"],
                     help="kernel path the library takes where it can run (default: the library's own choice)")
+    ap.add_argument("--op", default="fwd", choices=["fwd", "bwd"],
+                    help="bwd: time lot_attention_bwd (gradients of q, k, v, z, beta; one GPU) instead of the forward")
     ap.add_argument("--iters", type=int, default=None,
                     help="Sinkhorn iterations (default: the configuration's); 0 = apply passes only")
     return ap.parse_args()
@@ -388,10 +390,87 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_backward(args):
+    """The backward pass (Section "Learning") timed like the forward: CUDA events, L2 flushed between steps."""
+    import torch
+    from paper_2509_23436_b200 import binding as lot
+    from paper_2509_23436_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    x = workload(args)
+    B, H, n, d, r = x.shape
+    q, k, v, z, beta = (t.to(dev) for t in (x.q, x.k, x.v, x.z, x.beta))
+    key_len = None if x.key_len is None else x.key_len.to(dev)
+    dout = synth.cotangent(x).to(dev)
+    code = lot.LOT_BF16 if q.dtype == torch.bfloat16 else lot.LOT_F32
+    ws = torch.empty(max(256, lot.lot_bwd_workspace_bytes(B, H, n, d, r, code, x.iters)), device=dev, dtype=torch.uint8)
+    out = torch.empty_like(q)
+    fws = torch.empty(max(256, lot.lot_workspace_bytes(B, H, n, d, r, code)), device=dev, dtype=torch.uint8)
+    flush = torch.empty(512 << 20, device=dev, dtype=torch.uint8)
+    stream = torch.cuda.current_stream()
+
+    def bwd():
+        lot.lot_attention_bwd(q, k, v, z, beta, key_len, dout, x.eps, x.iters, ws=ws, stream=stream)
+
+    def fwd():
+        lot.lot_attention_fwd_ex(q, k, v, z, beta, key_len, x.eps, x.iters, out=out, ws=fws, stream=stream)
+
+    def timed(fn, steps):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        torch.cuda.synchronize()
+        for a, b in evs:
+            flush.fill_(0)
+            a.record(stream)
+            fn()
+            b.record(stream)
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs]
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        flush.fill_(1)
+        bwd()
+        fwd()
+    torch.cuda.synchronize()
+    if lot.lot_device_status(ws) != 0:
+        raise SystemExit("device status flagged during warm-up")
+    sampler = ClockSampler(0)
+    sampler.start()
+    tb = timed(bwd, args.steps)
+    clocks = sampler.finish()
+    tf = timed(fwd, args.steps)
+    ms = sum(tb) / len(tb)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    s_el = q.element_size()
+    abytes = B * H * n * d * 7 * s_el + 2 * H * r * (d + 1) * 4 + (B * 4 if key_len is not None else 0)
+    achieved = abytes / (ms * 1e-3) / 1e9
+    tdt = str(q.dtype).replace("torch.", "")
+    line = {"metric": "lot_attn_bwd_tokens_per_s", "value": B * n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": ARITH[0][tdt], "data": "synthetic",
+            "config": config_of(x, {"l2": "flushed between timed steps (512 MiB overwrite)",
+                                    "op": "backward (forward recomputed inside, materialised similarities)"}),
+            "clocks": clocks, "gpu_launches": (2 * x.iters + 15) * args.steps,
+            "forward_ms_per_step": sum(tf) / len(tf), "backward_over_forward": ms / (sum(tf) / len(tf)),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_source": peak_src, "algorithmic_bytes": abytes,
+                         "note": "q, k, v, dout read once; dq, dk, dv written once; z, beta, dz, dbeta"}}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse()
     if args.impl == "reference":
         run_reference(args)
+    elif args.op == "bwd":
+        run_backward(args)
     else:
         run_ours(args)
 

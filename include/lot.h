@@ -166,6 +166,10 @@ LOT_API size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype)
  *      column mass below 2^-80) is recomputed by the streamed kernels, which are launched behind it
  *      and return at once otherwise (device flag LOT_DEV_RECOMPUTED).  It can run many more shapes
  *      (lot_debug_hook what = 4), but measured no faster there.
+ *   3  the slice path (same tensors; n <= 512 and 16 ceil(n/16) x (r padded to 16, 32 or 64) <= 16384): one
+ *      thread block per (batch, head) slice keeps a side's logits in float32 registers for all iterations
+ *      (warp-level tensor-core products, shared memory for K, V, Q and the r x d intermediate); nothing
+ *      crosses thread blocks, no workspace beyond the status word.  Taken wherever it can run.
  * On paths 1 and 2 the potentials agree with an exact float evaluation to about 1e-4 and the output
  * to the bf16 rounding of `out`.
  */
@@ -217,7 +221,7 @@ LOT_API int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
  *   beta is treated as r free positive numbers per head (no simplex constraint: a softmax parametrisation is the
  *   caller's chain rule); dz and dbeta are summed over the batch.
  * The forward is recomputed (materialised similarities, general path arithmetic: float32 for bf16 tensors,
- * float64 for float32 tensors); only the pivot potentials of every iteration are kept.  2*iters + 20 launches.
+ * float64 for float32 tensors); only the pivot potentials of every iteration are kept.  2*iters + 15 kernel launches.
  * ws: lot_bwd_workspace_bytes(...) bytes of device scratch, 256-byte aligned, owned by the caller; the device
  * status word of the recomputed forward sits at its start (lot_device_status).
  * Errors as lot_attention_fwd_ex.  B == 0 or n == 0: dz and dbeta are zero-filled, nothing else is touched.

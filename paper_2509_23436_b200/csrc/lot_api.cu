@@ -187,16 +187,19 @@ void remember_ws(const void *ws, int path, unsigned tag, size_t fused_off)
     g_ws_records[ws] = WsRecord{path, tag, fused_off};
 }
 
-enum { kPathGeneral = 0, kPathStreamed = 1, kPathResident = 2 };
+enum { kPathGeneral = 0, kPathStreamed = 1, kPathResident = 2, kPathSlice = 3 };
 std::atomic<int> g_force_path{-1};      // test hook: 0 picks the general path, 1 or 2 that tensor-core path wherever it can run
 int choose_path(int dtype, int B, int H, int n, int d, int r)
 {
     if (!fused_supported(dtype, d, r)) return kPathGeneral;
     const bool res_ok = B >= 1 && n >= 1 && resident_geometry(dtype, B, H, n, d, r).ok;
+    const bool slice_ok = B >= 1 && slice_supported(dtype, n, d, r);
     const int force = g_force_path.load();
     if (force == kPathGeneral) return kPathGeneral;
     if (force == kPathStreamed) return kPathStreamed;
     if (force == kPathResident) return res_ok ? kPathResident : kPathStreamed;
+    // short sequences: one thread block per slice, everything on chip, exact float32 logits
+    if (slice_ok) return kPathSlice;
     // Measured on B200 (see the design notes): the resident kernel wins where the streamed one has no stored-kernel
     // passes (r <= 32, every pass recomputes logits and exponentials) and every thread block holds its whole share at
     // once (whole slices, one wave); elsewhere the streamed kernel is as fast or faster.
@@ -333,6 +336,7 @@ size_t lot_workspace_bytes(int B, int H, int n, int d, int r, int dtype)
     const int path = choose_path(dtype, B, H, n, d, r);
     if (path == kPathResident) return up256(resident_layout(B, H, n, d, r).total) + fused_layout(B, H, n, d, r).total;
     if (path == kPathStreamed) return fused_layout(B, H, n, d, r).total;
+    if (path == kPathSlice) return 256;                              // the status word
     return attn_layout(B, H, n, d, r, dtype).total;
 }
 
@@ -350,6 +354,7 @@ int lot_launch_count(int dtype, int B, int H, int n, int d, int r, int iters)
     const int path = lot_path(dtype, B, H, n, d, r, iters);
     if (path == kPathResident) return 1 + 2;                        // the two streamed kernels return at once unless asked to redo
     if (path == kPathStreamed) return fused_launches(B, H, n, r, iters);
+    if (path == kPathSlice) return 1;
     return 2 + iters + 1 + 2;
 }
 
@@ -380,6 +385,13 @@ int lot_attention_fwd_ex(const void *q, const void *k, const void *v,
         (key_len && (reinterpret_cast<uintptr_t>(key_len) & 3u)))
         return LOT_ERR_INVALID_ARG;
     const int path = choose_path(dtype, B, H, n, d, r);
+    if (path == kPathSlice) {
+        if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < 256) return LOT_ERR_WORKSPACE;
+        remember_ws(ws, kPathSlice, 0, 0);
+        cudaError_t e = slice_attention(q, k, v, z, beta, key_len, B, H, n, r, eps, iters, out, g1_out, g2_out,
+                                        at<int>(ws, 0), (cudaStream_t)stream);
+        return e == cudaSuccess ? LOT_OK : LOT_ERR_CUDA;
+    }
     if (path != kPathGeneral) {
         const size_t res_bytes = path == kPathResident ? up256(resident_layout(B, H, n, d, r).total) : 0;
         const size_t need = res_bytes + fused_layout(B, H, n, d, r).total;

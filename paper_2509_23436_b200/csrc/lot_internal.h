@@ -147,6 +147,12 @@ cudaError_t resident_attention(const void *q, const void *k, const void *v, cons
                                void *out, float *g1_out, float *g2_out, void *ws, unsigned *tag_out, cudaStream_t st);
 void resident_debug(int what, long long value);
 
+// ---- slice path (lot_slice.cu): bf16 tensors, d = 64, r <= 64, short sequences; one thread block per slice ----
+bool slice_supported(int dtype, int n, int d, int r);
+cudaError_t slice_attention(const void *q, const void *k, const void *v, const float *z, const float *beta,
+                            const int32_t *key_len, int B, int H, int n, int r, float eps, int iters, void *out,
+                            float *g1_out, float *g2_out, int *status, cudaStream_t st);
+
 // ---- apply stages from the stored Gibbs kernel (lot_apply.cu), behind the streamed Sinkhorn kernel ----
 size_t stored_apply_wpart_bytes(int B, int H, int n);
 cudaError_t stored_apply(const void *kt, int npad, const float *G, const float *beta, const int32_t *key_len, const int *decision,

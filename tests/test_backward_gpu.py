@@ -58,10 +58,28 @@ def oracle_grads(x, dout):
     return dq, dk, dv, dz, dbeta
 
 
+# config 5's peaked similarities (Gaussian-mixture queries and keys, d = 128), small eps
+PEAKED = [
+    (1, 2, 1024, 128, 64, 5, 0.05, BF16),
+    (1, 1, 512, 128, 16, 20, 0.01, F32),
+    (2, 1, 640, 128, 256, 5, 0.1, F32),
+]
+
+
+@pytest.mark.parametrize("B,H,n,d,r,iters,eps,dtype", PEAKED)
+def test_backward_peaked_costs(B, H, n, d, r, iters, eps, dtype):
+    run_case(synth.make(B, H, n, d, r, seed=7500 + n + r, dtype=dtype, eps=eps, iters=iters, qk="mixture"), False)
+
+
 @pytest.mark.parametrize("B,H,n,d,r,iters,eps,dtype,masked", CASES)
 def test_backward_matches_oracle(B, H, n, d, r, iters, eps, dtype, masked):
-    x = synth.make(B, H, n, d, r, seed=7100 + n + r, dtype=dtype, eps=eps, iters=iters,
-                   key_len_range=(n // 2, n) if masked else None)
+    run_case(synth.make(B, H, n, d, r, seed=7100 + n + r, dtype=dtype, eps=eps, iters=iters,
+                        key_len_range=(n // 2, n) if masked else None), masked)
+
+
+def run_case(x, masked):
+    B, H, n, d, r = x.shape
+    eps, iters, dtype = x.eps, x.iters, x.q.dtype
     dout = synth.cotangent(x)
     dev = torch.device("cuda:0")
     kl = None if x.key_len is None else x.key_len.to(dev)

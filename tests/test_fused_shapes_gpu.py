@@ -6,10 +6,20 @@ import numpy as np
 import pytest
 import torch
 
+from paper_2509_23436_b200 import binding as lot
 from paper_2509_23436_b200 import synth
 from lot_testutil import check_slice, gpu_forward, oracle_slice
 
 pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def streamed_path():
+    """Short sequences take the slice path by default: these cases are about the streamed kernels' geometries."""
+    lot.lot_debug_hook(4, 1)
+    yield
+    lot.lot_debug_hook(4, -1)
+
 
 CASES = [
     # B, H, n, r, iters, eps, key mask
