@@ -224,10 +224,12 @@ def run_reference(args):
 # --------------------------------------------------------------------------- our arm
 PATH_NAMES = {0: "general path (cost, T+1 Sinkhorn passes, two apply kernels)",
               1: "fused_forward_kernel (persistent, Gibbs kernel streamed from L2; plus the pivot preparation)",
-              2: "resident_forward_kernel (persistent, Gibbs kernel resident in shared memory and TMEM)"}
+              2: "resident_forward_kernel (persistent, Gibbs kernel resident in shared memory and TMEM)",
+              3: "slice_forward_kernel (one thread block per slice, logits and Gibbs kernel in float32 registers)"}
 ARITH = {0: {"bfloat16": "f32", "float32": "f64"},
          1: {"bfloat16": "bf16 operands, f32 accumulate, bf16 stored Gibbs kernel"},
-         2: {"bfloat16": "bf16 operands, f32 accumulate, bf16 resident Gibbs kernel"}}
+         2: {"bfloat16": "bf16 operands, f32 accumulate, bf16 resident Gibbs kernel"},
+         3: {"bfloat16": "bf16 operands, f32 accumulate, f32 Gibbs kernel in registers"}}
 
 
 def run_ours(args):

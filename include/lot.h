@@ -77,6 +77,8 @@ enum lot_device_flag {
     LOT_DEV_NONFINITE = 1, /* a pivot potential became inf/nan (e.g. beta_t <= 0) */
     LOT_DEV_EMPTY = 2,     /* a key_len entry was <= 0: that slice has no key mass; its output is zeros */
     LOT_DEV_TIMEOUT = 4,   /* a bounded device-side wait gave up; results of the call are invalid */
+    LOT_DEV_BOUNDS = 16,   /* bounds-check build only (compiled with -DLOT_DEBUG, lot_version() = 100100): an index of a
+                              general-path or backward kernel fell outside its buffer; the access was skipped */
     LOT_DEV_RECOMPUTED = 8 /* information only: the resident path could not represent the problem (see lot_path)
                               and the streamed kernels recomputed the call; the results are valid */
 };

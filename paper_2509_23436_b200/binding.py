@@ -15,9 +15,10 @@ import torch
 
 LOT_F32, LOT_BF16 = 0, 1
 LOT_OK = 0
-LOT_DEV_NONFINITE, LOT_DEV_EMPTY, LOT_DEV_TIMEOUT, LOT_DEV_RECOMPUTED = 1, 2, 4, 8
+LOT_DEV_NONFINITE, LOT_DEV_EMPTY, LOT_DEV_TIMEOUT, LOT_DEV_RECOMPUTED, LOT_DEV_BOUNDS = 1, 2, 4, 8, 16
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblot.so")
+# LOT_LIBRARY selects another build of the same library (the bounds-check build liblot_debug.so)
+_LIB_PATH = os.environ.get("LOT_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblot.so")
 _lib = None
 
 _vp, _i, _f, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t

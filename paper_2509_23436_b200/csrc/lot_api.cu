@@ -220,7 +220,11 @@ std::mutex g_static_mu;
 
 extern "C" {
 
+#ifdef LOT_DEBUG
+int lot_version(void) { return 100 + 100000; }      // the bounds-check build answers 100100
+#else
 int lot_version(void) { return 100; }
+#endif
 
 const char *lot_status_string(int status)
 {
@@ -603,6 +607,7 @@ int lot_device_status(const void *ws, lot_stream_t stream, int *status)
     if (rec.path != kPathResident) {
         if (cudaMemcpyAsync(status, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOT_ERR_CUDA;
         if (cudaStreamSynchronize(s) != cudaSuccess) return LOT_ERR_CUDA;
+        if (kernels_debug_flag() | backward_debug_flag()) *status |= LOT_DEV_BOUNDS;      // bounds-check build only
         return LOT_OK;
     }
     // resident path: {flags | tag << 32, redo word} at the start, the streamed kernels' word behind the resident block

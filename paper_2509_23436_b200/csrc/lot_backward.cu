@@ -121,7 +121,7 @@ bwd_row_kernel(BwdRowArgs a)
         for (int v = 0; v < NV; ++v) {
             const int t = (v * LPR + cl) * 4;
             LT cc[4] = {(LT)0, (LT)0, (LT)0, (LT)0}, xx[4] = {(LT)0, (LT)0, (LT)0, (LT)0};
-            if (rv && t < r) {
+            if (rv && t < r && LOT_CHECK((size_t)i * r + (vec ? t + 4 : t + 1) <= (size_t)a.n * r)) {
                 load_row4<LT>(C + (size_t)i * r + t, vec, t, r, cc);
                 load_row4<LT>(D + (size_t)i * r + t, vec, t, r, xx);
             }
@@ -185,7 +185,7 @@ bwd_row_kernel(BwdRowArgs a)
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
                 const int t = (v * LPR + cl) * 4;
-                if (t < r) {
+                if (t < r && LOT_CHECK((size_t)i * r + (vec ? t + 4 : t + 1) <= (size_t)a.n * r)) {
                     LT xx[4] = {x[v * 4], x[v * 4 + 1], x[v * 4 + 2], x[v * 4 + 3]};
                     store_row4<LT>(D + (size_t)i * r + t, vec, t, r, xx);
                 }
@@ -315,7 +315,7 @@ gemm_nt_kernel(const AT *__restrict__ A, const float *__restrict__ Bm, OutT *__r
 #pragma unroll
         for (int y = 0; y < 4; ++y) {
             const int j = j0 + tx * 4 + y;
-            if (j < J) ob[(size_t)i * J + j] = StoreAs<OutT>::conv(acc[x][y]);
+            if (j < J && LOT_CHECK((size_t)i * J + j < (size_t)n * J)) ob[(size_t)i * J + j] = StoreAs<OutT>::conv(acc[x][y]);
         }
     }
 }
@@ -420,7 +420,7 @@ bwd_dz_part_kernel(const LT *__restrict__ dC, const T *__restrict__ q, const T *
 #pragma unroll
         for (int y = 0; y < 4; ++y) {
             const int c = c0 + tx * 4 + y;
-            if (c < d) pp[(size_t)t * d + c] = acc[x][y];
+            if (c < d && LOT_CHECK((size_t)t * d + c < (size_t)r * d)) pp[(size_t)t * d + c] = acc[x][y];
         }
     }
 }
@@ -525,5 +525,7 @@ cudaError_t launch_bwd_dz(const void *dC, const void *q, const void *k, int dtyp
                                                           static_cast<const float *>(dbeta_acc), dz, dbeta, B, H, d, r, chunks);
     return cudaGetLastError();
 }
+
+LOT_DEBUG_FLAG_READER(backward_debug_flag)
 
 } // namespace lot

@@ -11,6 +11,25 @@
 #include <math.h>
 #include <stdint.h>
 
+// Bounds-check build (-DLOT_DEBUG): every checked global access states the extent of its buffer; an access outside it
+// is skipped and recorded in a per-file device word that lot_device_status reports as LOT_DEV_BOUNDS.  Never a trap.
+#ifdef LOT_DEBUG
+static __device__ int g_lot_bounds_flag;
+#define LOT_CHECK(cond) ((cond) ? true : (atomicOr(&g_lot_bounds_flag, 1), false))
+#define LOT_DEBUG_FLAG_READER(name)                                                              \
+    int name()                                                                                   \
+    {                                                                                            \
+        int v = 0, zero = 0;                                                                     \
+        if (cudaMemcpyFromSymbol(&v, g_lot_bounds_flag, sizeof(int)) != cudaSuccess) return 0;   \
+        (void)cudaMemcpyToSymbol(g_lot_bounds_flag, &zero, sizeof(int));                         \
+        return v;                                                                                \
+    }
+#else
+#define LOT_CHECK(cond) true
+#define LOT_DEBUG_FLAG_READER(name) \
+    int name() { return 0; }
+#endif
+
 namespace lot {
 
 constexpr float kLog2e = 1.4426950408889634f;

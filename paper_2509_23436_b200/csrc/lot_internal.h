@@ -58,6 +58,10 @@ struct ApplyArgs {
     double scale_d;
 };
 
+// bounds-check build only (0 otherwise): reads and clears the file's record of skipped out-of-range accesses
+int kernels_debug_flag();
+int backward_debug_flag();
+
 int pass_chunks(int nprob, int n);
 int apply_chunks(int BH, int n, int r, int d);
 

@@ -35,8 +35,10 @@ cost_kernel(const T *__restrict__ x, const float *__restrict__ z, OutT *__restri
             int idx = threadIdx.x + rep * 256;
             int row = idx / 8, k4 = (idx % 8) * 4;
             float xv[4] = {0.f, 0.f, 0.f, 0.f}, zv[4] = {0.f, 0.f, 0.f, 0.f};
-            if (i0 + row < n && k0 + k4 < d) load4(xb + (size_t)(i0 + row) * d + k0 + k4, xv);
-            if (t0 + row < r && k0 + k4 < d) load4(zb + (size_t)(t0 + row) * d + k0 + k4, zv);
+            if (i0 + row < n && k0 + k4 < d && LOT_CHECK((size_t)(i0 + row) * d + k0 + k4 + 4 <= (size_t)n * d))
+                load4(xb + (size_t)(i0 + row) * d + k0 + k4, xv);
+            if (t0 + row < r && k0 + k4 < d && LOT_CHECK((size_t)(t0 + row) * d + k0 + k4 + 4 <= (size_t)r * d))
+                load4(zb + (size_t)(t0 + row) * d + k0 + k4, zv);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 Xs[k4 + j][row] = (AccT)xv[j];
@@ -64,7 +66,7 @@ cost_kernel(const T *__restrict__ x, const float *__restrict__ z, OutT *__restri
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
             int t = t0 + tx * 4 + b;
-            if (t < r) cb[(size_t)i * r + t] = (OutT)acc[a][b];
+            if (t < r && LOT_CHECK((size_t)i * r + t < (size_t)n * r)) cb[(size_t)i * r + t] = (OutT)acc[a][b];
         }
     }
 }
@@ -99,22 +101,6 @@ cudaError_t launch_cost(const void *x, const float *z, int dtype, int BH, int H,
 // merged lane -> warp -> block -> grid in a fixed order.
 // FINAL = closing token update: writes M (and optionally g, f, plan), no pivot update.
 // ------------------------------------------------------------------------------------
-// Add one term to a column pair.  The term is given twice: as the plain product `term` = 2^x (which may have
-// underflowed to zero) and as its exponent x.  While the pair's reference exponent kap is above -100, term * 2^-kap
-// equals 2^(x - kap) to rounding, and a term lost to underflow (x < -126) is below 2^-26 of the reference, less than
-// the sum can resolve: no exponential is needed.  A term more than 2^20 above the reference, or a reference outside
-// that range (phi is NaN then, and the comparison fails), takes the exact update and renews phi.
-__device__ __forceinline__ void col_add(float &kap, float &phi, float &S, float term, float x)
-{
-    const float t = term * phi;
-    if (t <= 1048576.f) {
-        S += t;
-    } else if (x > neg_inf()) {
-        pair_add(kap, S, x);
-        phi = kap >= -100.f ? ex2(-kap) : __int_as_float(0x7fc00000);
-    }
-}
-
 constexpr int kPassWarps = 8;
 constexpr int kRowsPerThread = 2;
 
@@ -150,7 +136,7 @@ __device__ __forceinline__ void load_cost4<double>(const double *p, bool vec, in
 // in (float for bf16 tensors; double when the caller's tensors are float32, so that logits of
 // magnitude ~1e3 at small eps keep an absolute accuracy well below the 1e-4 output tolerance).
 template <int LPR, int NV, bool FINAL, typename CostT, typename LT>
-__global__ void __launch_bounds__(kPassWarps * 32, 2)
+__global__ void __launch_bounds__(kPassWarps * 32)
 sinkhorn_pass_kernel(PassArgs a)
 {
     __shared__ float sm_k[kPassWarps][256];
@@ -174,15 +160,12 @@ sinkhorn_pass_kernel(PassArgs a)
     const float *mass_p = a.mass ? a.mass + (size_t)p * a.n : nullptr;
 
     LT Gk[CPL];
-    // column sums as pairs (kap, S) = S * 2^kap; phi = 2^-kap while kap is in the range where plain products can
-    // stand in for the exponential of the difference (see col_add), NaN otherwise
-    float kap[CPL], phi[CPL], S[CPL];
+    float kap[CPL], S[CPL];
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
         const int t = ((k >> 2) * LPR + cl) * 4 + (k & 3);
         Gk[k] = t < r ? Gp[t] : (LT)neg_inf();        // columns beyond r: logit -inf, term 0
         kap[k] = neg_inf();
-        phi[k] = t < r ? __int_as_float(0x7fc00000) : 0.f;
         S[k] = 0.f;
     }
     const int row0 = chunk * a.rows_per_chunk;
@@ -205,7 +188,8 @@ sinkhorn_pass_kernel(PassArgs a)
             for (int v = 0; v < NV; ++v) {
                 const int t = (v * LPR + cl) * 4;
                 CostT cc[4] = {(CostT)0, (CostT)0, (CostT)0, (CostT)0};
-                if (rv[u] && t < r) load_cost4<CostT>(C + (size_t)i * r + t, vec, t, r, cc);
+                if (rv[u] && t < r && LOT_CHECK((size_t)i * r + (vec ? t + 4 : t + 1) <= (size_t)a.n * r))
+                    load_cost4<CostT>(C + (size_t)i * r + t, vec, t, r, cc);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) c[u][v * 4 + j] = cc[j];
             }
@@ -223,13 +207,12 @@ sinkhorn_pass_kernel(PassArgs a)
             }
 #pragma unroll
             for (int off = LPR / 2; off > 0; off >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, off));
-            float e[CPL], pe[CPL];
+            float e[CPL];
             float s = 0.f;
 #pragma unroll
             for (int k = 0; k < CPL; ++k) {
                 e[k] = (float)(l[k] - m);          // <= 0, exact difference of nearby logits
-                pe[k] = ex2(e[k]);
-                s += pe[k];
+                s += ex2(e[k]);
             }
 #pragma unroll
             for (int off = LPR / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
@@ -237,9 +220,9 @@ sinkhorn_pass_kernel(PassArgs a)
             if (!FINAL) {
                 if (rv[u]) {
                     const float shift = mass_p != nullptr ? lmi - lgs : -lgs;
-                    const float wrow = mass_p != nullptr ? mi[u] * __fdividef(1.f, s) : __fdividef(1.f, s);
 #pragma unroll
-                    for (int k = 0; k < CPL; ++k) col_add(kap[k], phi[k], S[k], pe[k] * wrow, e[k] + shift);
+                    for (int k = 0; k < CPL; ++k)
+                        if (e[k] > neg_inf()) pair_add(kap[k], S[k], e[k] + shift);
                 }
             } else if (i < row_end) {
                 if (cl == 0) {
@@ -544,7 +527,7 @@ apply_out_kernel(ApplyArgs a)
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
         int i = i0 + ty * 4 + x, c = c0 + tx * 4;
-        if (i < n && c < d) store4(O + (size_t)i * d + c, acc[x]);
+        if (i < n && c < d && LOT_CHECK((size_t)i * d + c + 4 <= (size_t)n * d)) store4(O + (size_t)i * d + c, acc[x]);
     }
 }
 
@@ -669,5 +652,7 @@ cudaError_t launch_cls_row(const void *q, const void *k, const void *v, const in
                                                              scores, static_cast<__nv_bfloat16 *>(out));
     return cudaGetLastError();
 }
+
+LOT_DEBUG_FLAG_READER(kernels_debug_flag)
 
 } // namespace lot

@@ -296,16 +296,24 @@ __device__ __forceinline__ void solve(float (&L)[MT][NT][4], float (&G)[NT][2], 
                 const float tot = block_columns<NT, false>(c, sRed, warp, lane);
                 float g_old = 0.f;
                 const bool ok = tot >= kTiny;
-                if (tid < r) {
-                    g_old = sG[tid];
-                    if (ok) {
-                        const float gn = sLb[tid] + Gmax - lg2(tot);
-                        sG[tid] = gn;
-                        atomicMax(sStat + ((it + 1) & 1) * 2, enc_ord(gn));
-                        atomicMin(sStat + ((it + 1) & 1) * 2 + 1, enc_ord(gn));
-                        if (!isfinite(gn)) atomicOr(status, 1 /* LOT_DEV_NONFINITE */);
-                    } else {
-                        *sFlag = 1;
+                if (warp < 2) {                                    // threads 0..63 own the columns
+                    uint32_t emax = 0u, emin = 0xffffffffu;
+                    if (tid < r) {
+                        g_old = sG[tid];
+                        if (ok) {
+                            const float gn = sLb[tid] + Gmax - lg2(tot);
+                            sG[tid] = gn;
+                            emax = emin = enc_ord(gn);
+                            if (!isfinite(gn)) atomicOr(status, 1 /* LOT_DEV_NONFINITE */);
+                        } else {
+                            *sFlag = 1;
+                        }
+                    }
+                    emax = __reduce_max_sync(0xffffffffu, emax);
+                    emin = __reduce_min_sync(0xffffffffu, emin);
+                    if (lane == 0) {
+                        atomicMax(sStat + ((it + 1) & 1) * 2, emax);
+                        atomicMin(sStat + ((it + 1) & 1) * 2 + 1, emin);
                     }
                 }
                 if (tid == 0) { sStat[(it & 1) * 2] = 0u; sStat[(it & 1) * 2 + 1] = 0xffffffffu; }
@@ -478,6 +486,9 @@ slice_forward_kernel(const SliceParams P)
     };
     load_rows(P.k + tok, sX);
     load_rows(P.v + tok, sV);
+    // the query rows are wanted after the key side is solved: have them in L2 by then
+    for (int idx = threadIdx.x; idx < n; idx += kThreads)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(P.q + tok + (size_t)idx * kD));
     // pivots of this head, scaled to base-2 logit units, as bf16 hi + lo
     for (int idx = threadIdx.x; idx < PL::RP * (kD / 2); idx += kThreads) {
         const int t = idx / (kD / 2), c2 = (idx % (kD / 2)) * 2;
