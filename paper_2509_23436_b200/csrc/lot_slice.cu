@@ -3,13 +3,13 @@
 // n <= 512, 16 ceil(n/16) x rpad <= 16384).  Nothing crosses thread blocks and nothing but the inputs and the output
 // touches global memory:
 //   key side:   K, V -> shared memory; logits L2 = K Z^T * log2(e)/eps on the tensor cores (warp-level MMA, Z as bf16
-//               hi + lo) into registers; T log-domain Sinkhorn iterations on the registers (row reductions inside a
-//               lane quad, column sums through shared memory in a fixed order); plan rows -> shared memory as bf16
-//               hi + lo; W = Gamma2^T V on the tensor cores; W' = Diag(1/beta) W -> shared memory, bf16 hi + lo.
+//               hi + lo) into registers; T Sinkhorn iterations on the registers (scaling form on the float32 Gibbs
+//               kernel, log domain when the potentials spread too far; row reductions inside a lane quad, column
+//               sums through shared memory in a fixed order); plan rows -> shared memory as bf16 hi + lo;
+//               W = Gamma2^T V on the tensor cores; W' = Diag(1/beta) W -> shared memory, bf16 hi + lo.
 //   query side: Q -> shared memory; logits; iterations; out = R1 W' with the plan rows straight from the registers
 //               that held the logits (an accumulator fragment is an A fragment); bf16 rows to global memory.
-// The logits stay exact float32 for all iterations: no stored bf16 Gibbs kernel, no range limit.  A column sum that
-// underflows in plain float32 (a pivot no token is near) is recomputed relative to its column maximum.
+// Logits and Gibbs kernel are float32 in registers: no stored bf16 kernel, and no range limit (see solve).
 // 512 threads; warp w owns the 16-row tiles w, w + 16; a thread holds rows g and g + 8 (g = lane / 4) of each and,
 // per 8-column tile, columns 2 (lane % 4) and + 1: the accumulator layout of mma.m16n8k16.
 #include "lot_common.cuh"
